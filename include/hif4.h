@@ -1,0 +1,139 @@
+/*
+ * hif4.h -- C ABI of the HiF4 (HiFloat4) W4A4 linear-layer hot path for NVIDIA B200 (sm_100a).
+ *
+ * HiF4 is the 4-bit block floating-point format of "HiFloat4 Format for Language Model
+ * Inference" (Section II).  One HiF4 *unit* stores 64 values in 288 bits: 32 bits of shared
+ * three-level scaling metadata plus 64 four-bit sign-magnitude S1P2 elements (Section II-A,
+ * Table I, Table II: 4.5 bits per value).
+ *
+ * ---------------------------------------------------------------------------------------------
+ * Unit layout in memory (36 bytes, 4-byte aligned, units of a row consecutive, rows consecutive).
+ * The paper's figure of the unit is not reproduced in its text, so this byte order is a
+ * convention of this library:
+ *
+ *   bytes 0..3   little-endian uint32 `meta`
+ *                  bits  7:0   E6M2 level-1 scale byte `eeeeee mm` (Table I): value
+ *                              2^(e-48) * (1 + m/4); 0xFF is NaN, there is no zero or infinity
+ *                  bits 15:8   E1_8  level-2 micro-exponents, bit 8+j  covers elements 8j..8j+7
+ *                  bits 31:16  E1_16 level-3 micro-exponents, bit 16+k covers elements 4k..4k+3
+ *   bytes 4..35  S1P2 codes, element i in byte 4 + i/2, low nibble for even i, high nibble for
+ *                odd i; nibble = sign<<3 | magnitude, magnitude m in 0..7 meaning m/4.
+ *
+ * Value of element i (Eq. 2, 0-based indices):
+ *   V_i = (-1)^sign * (m/4) * 2^(E1_8[i/8] + E1_16[i/4]) * E6M2,   all 64 are NaN if E6M2 is NaN.
+ * ---------------------------------------------------------------------------------------------
+ *
+ * Conventions common to every call
+ *   - All data pointers are DEVICE pointers unless a parameter says "host".  The caller owns every
+ *     buffer; the library never allocates, frees or synchronises (hif4_last_device_status is the
+ *     one documented exception and synchronises the stream it is given).
+ *   - Every call is asynchronous on `stream` (a cudaStream_t passed as void* so that this header
+ *     needs no CUDA header; NULL is the legacy default stream).
+ *   - The return value is a status code.  Argument errors are found on the host before any launch.
+ *     NaN and Inf in the data are not errors; they encode as the format defines.
+ *   - Matrices are row-major.  Both GEMM operands are quantised along K (units contiguous in K),
+ *     because Eq. 3 pairs unit k of a row of A with unit k of a row of B.  A weight W[K_in, N_out]
+ *     is therefore handed over as its transpose [N, K].
+ */
+#ifndef HIF4_H_
+#define HIF4_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HIF4_UNIT_ELEMS 64   /* elements per unit (Section II-A)                    */
+#define HIF4_UNIT_BYTES 36   /* 4 metadata bytes + 32 code bytes = 288 bits         */
+
+typedef enum {
+  HIF4_OK = 0,
+  HIF4_ERR_NULL = 1,           /* a required pointer is NULL                                   */
+  HIF4_ERR_SHAPE = 2,          /* negative size, cols or K not a multiple of 64, ld too small  */
+  HIF4_ERR_ALIGN = 3,          /* pointer or leading dimension breaks the stated alignment     */
+  HIF4_ERR_DTYPE = 4,          /* unknown hif4_dtype / hif4_round value                        */
+  HIF4_ERR_WORKSPACE = 5,      /* workspace smaller than hif4_*_workspace reports              */
+  HIF4_ERR_CUDA = 6,           /* a CUDA call or launch failed; cudaGetLastError keeps the code*/
+  HIF4_ERR_DEVICE_TIMEOUT = 7, /* a bounded wait inside a kernel ran out (see last_device_status) */
+  HIF4_ERR_UNSUPPORTED = 8     /* valid request that this build does not implement             */
+} hif4_status;
+
+typedef enum { HIF4_BF16 = 0, HIF4_FP32 = 1 } hif4_dtype;
+
+/* Rounding used where Algorithm 1 rounds to E6M2 and to S1P2 ("round-half-to-even or
+ * round-half-away-from-zero", Section II-B).  Products inside the algorithm always round to
+ * nearest-even.  */
+typedef enum { HIF4_RNE = 0, HIF4_RHA = 1 } hif4_round;
+
+/* Bytes of the packed form of a [rows, cols] matrix: rows * (cols/64) * 36 (Section II-A).
+ * Returns 0 when cols is not a multiple of 64 or a size is negative.  Host-only, no GPU use.  */
+size_t hif4_packed_bytes(int64_t rows, int64_t cols);
+
+/* hif4_quantize -- Algorithm 1 (Section II-B) applied to every 64-element unit of a matrix.
+ *   src        device, [rows, cols] of `dt`, row stride `ld_src` ELEMENTS (>= cols); base and row
+ *              stride must keep every row 16-byte aligned.
+ *   dst_units  device, rows*(cols/64) units of 36 bytes, row-major, 4-byte aligned (16-byte aligned
+ *              storage gives the fastest stores).  Fully overwritten.
+ *   mode       HIF4_RNE or HIF4_RHA.
+ * The working precision of the algorithm is that of the source type (BF16 arithmetic for BF16
+ * input, FP32 arithmetic for FP32 input).  A unit holding a NaN becomes the canonical NaN unit
+ * (meta 0x000000FF, codes 0).  rows == 0 or cols == 0 is a no-op returning HIF4_OK.  */
+hif4_status hif4_quantize(const void* src, hif4_dtype dt, int64_t rows, int64_t cols,
+                          int64_t ld_src, void* dst_units, hif4_round mode, void* stream);
+
+/* hif4_dequantize -- Eq. 2 for every element; exact in BF16 and FP32.
+ *   src_units  device, rows*(cols/64) units, 4-byte aligned.
+ *   dst        device, [rows, cols] of `dt`, row stride `ld_dst` elements (>= cols), rows 16-byte
+ *              aligned.  Fully overwritten inside [rows, cols]; padding beyond cols is untouched.  */
+hif4_status hif4_dequantize(const void* src_units, int64_t rows, int64_t cols, void* dst,
+                            hif4_dtype dt, int64_t ld_dst, void* stream);
+
+/* Workspace (device scratch) that hif4_gemm needs for this shape; may be 0.  Host-only.  */
+hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size_t* bytes);
+
+/* hif4_gemm -- C = A * B^T with A, B in HiF4 and FP32 accumulation: C[i][j] is the sum over the
+ * K/64 unit pairs of Eq. 3's dot product of unit k of row i of A with unit k of row j of B.
+ *   A_units    device, [M, K/64] units.        B_units  device, [N, K/64] units.
+ *   C          device, [M, N] FP32, row stride `ldc` elements (>= N), 16-byte aligned rows
+ *              (ldc % 4 == 0).  Overwritten (no alpha/beta).
+ *   workspace  device scratch of at least hif4_gemm_workspace bytes, 256-byte aligned, contents
+ *              undefined on entry and exit; may be NULL when 0 bytes are needed.
+ * K must be a multiple of 64.  M == 0 or N == 0 is a no-op; K == 0 zero-fills C.
+ * Units whose E6M2 byte is NaN make every C entry they touch NaN.  */
+hif4_status hif4_gemm(const void* A_units, const void* B_units, float* C, int64_t M, int64_t N,
+                      int64_t K, int64_t ldc, void* workspace, size_t workspace_bytes,
+                      void* stream);
+
+hif4_status hif4_grouped_gemm_workspace(int num_groups, int64_t total_rows, int64_t N, int64_t K,
+                                        size_t* bytes);
+
+/* hif4_grouped_gemm -- the same contraction per group g (an MoE expert, Section IV-B converts the
+ * MoE linears):  C[off[g]:off[g+1], :] = A[off[g]:off[g+1], :] * B[g]^T.
+ *   A_units            device, [total_rows, K/64] units, rows sorted by group.
+ *   B_units            device, [num_groups, N, K/64] units.
+ *   C                  device, [total_rows, N] FP32, row stride ldc.
+ *   group_offsets_dev  device, num_groups+1 int64 prefix sums, off[0] = 0, off[num_groups] =
+ *                      total_rows, non-decreasing.  Read by the kernel only: routing results never
+ *                      return to the host.  Empty groups are allowed.  */
+hif4_status hif4_grouped_gemm(const void* A_units, const void* B_units, float* C,
+                              const int64_t* group_offsets_dev, int num_groups, int64_t total_rows,
+                              int64_t N, int64_t K, int64_t ldc, void* workspace,
+                              size_t workspace_bytes, void* stream);
+
+/* Synchronises `stream` and returns HIF4_ERR_DEVICE_TIMEOUT if any kernel of this library gave up
+ * a bounded wait since the last call (the flag is cleared), HIF4_ERR_CUDA if the stream reports
+ * an error, else HIF4_OK.  For tests and debugging.  */
+hif4_status hif4_last_device_status(void* stream);
+
+/* Static, NUL-terminated description of a status code.  Host-only.  */
+const char* hif4_status_string(hif4_status s);
+
+/* Number of kernels this library has launched in this process (monotonic, host-side counter).  */
+uint64_t hif4_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HIF4_H_ */
