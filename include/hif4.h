@@ -96,8 +96,9 @@ hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size_t* bytes);
 /* hif4_gemm -- C = A * B^T with A, B in HiF4 and FP32 accumulation: C[i][j] is the sum over the
  * K/64 unit pairs of Eq. 3's dot product of unit k of row i of A with unit k of row j of B.
  *   A_units    device, [M, K/64] units.        B_units  device, [N, K/64] units.
- *   C          device, [M, N] FP32, row stride `ldc` elements (>= N), 16-byte aligned rows
- *              (ldc % 4 == 0).  Overwritten (no alpha/beta).
+ *   C          device, [M, N] FP32, row stride `ldc` elements (>= N), 4-byte aligned; 16-byte
+ *              aligned rows (base % 16 == 0 and ldc % 4 == 0) allow vector stores.  Overwritten
+ *              inside [M, N] (no alpha/beta); padding beyond N is untouched.
  *   workspace  device scratch of at least hif4_gemm_workspace bytes, 256-byte aligned, contents
  *              undefined on entry and exit; may be NULL when 0 bytes are needed.
  * K must be a multiple of 64.  M == 0 or N == 0 is a no-op; K == 0 zero-fills C.

@@ -1,0 +1,72 @@
+// hif4_gemm / hif4_grouped_gemm entry points: argument checks on the host, then kernel selection.
+#include "hif4_common.cuh"
+#include "hif4_gemm_internal.cuh"
+
+using namespace hif4;
+
+namespace {
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+hif4_status check_common(const void* A, const void* B, const float* C, int64_t M, int64_t N, int64_t K,
+                         int64_t ldc) {
+  if (M < 0 || N < 0 || K < 0 || K % kUnitElems != 0 || ldc < N) return HIF4_ERR_SHAPE;
+  if (M == 0 || N == 0) return HIF4_OK;
+  if (!C || (K > 0 && (!A || !B))) return HIF4_ERR_NULL;
+  if (!aligned(A, 4) || !aligned(B, 4) || !aligned(C, 4)) return HIF4_ERR_ALIGN;
+  return HIF4_OK;
+}
+}  // namespace
+
+extern "C" hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size_t* bytes) {
+  if (!bytes) return HIF4_ERR_NULL;
+  if (M < 0 || N < 0 || K < 0 || K % kUnitElems != 0) return HIF4_ERR_SHAPE;
+  *bytes = 0;
+  return HIF4_OK;
+}
+
+extern "C" hif4_status hif4_gemm(const void* A_units, const void* B_units, float* C, int64_t M, int64_t N,
+                                 int64_t K, int64_t ldc, void* workspace, size_t workspace_bytes,
+                                 void* stream) {
+  (void)workspace;
+  (void)workspace_bytes;
+  const hif4_status chk = check_common(A_units, B_units, C, M, N, K, ldc);
+  if (chk != HIF4_OK || M == 0 || N == 0) return chk;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (K == 0) {
+    if (cudaMemset2DAsync(C, static_cast<size_t>(ldc) * 4, 0, static_cast<size_t>(N) * 4,
+                          static_cast<size_t>(M), st) != cudaSuccess)
+      return HIF4_ERR_CUDA;
+    return HIF4_OK;
+  }
+  return launch_gemm_simt(A_units, B_units, C, M, N, K, ldc, st);
+}
+
+extern "C" hif4_status hif4_grouped_gemm_workspace(int num_groups, int64_t total_rows, int64_t N, int64_t K,
+                                                   size_t* bytes) {
+  if (!bytes) return HIF4_ERR_NULL;
+  if (num_groups < 0 || total_rows < 0 || N < 0 || K < 0 || K % kUnitElems != 0) return HIF4_ERR_SHAPE;
+  *bytes = 0;
+  return HIF4_OK;
+}
+
+extern "C" hif4_status hif4_grouped_gemm(const void* A_units, const void* B_units, float* C,
+                                         const int64_t* group_offsets_dev, int num_groups, int64_t total_rows,
+                                         int64_t N, int64_t K, int64_t ldc, void* workspace,
+                                         size_t workspace_bytes, void* stream) {
+  (void)workspace;
+  (void)workspace_bytes;
+  if (num_groups < 0) return HIF4_ERR_SHAPE;
+  const hif4_status chk = check_common(A_units, B_units, C, total_rows, N, K, ldc);
+  if (chk != HIF4_OK || total_rows == 0 || N == 0 || num_groups == 0) return chk;
+  if (!group_offsets_dev) return HIF4_ERR_NULL;
+  if (!aligned(group_offsets_dev, 8)) return HIF4_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (K == 0) {
+    if (cudaMemset2DAsync(C, static_cast<size_t>(ldc) * 4, 0, static_cast<size_t>(N) * 4,
+                          static_cast<size_t>(total_rows), st) != cudaSuccess)
+      return HIF4_ERR_CUDA;
+    return HIF4_OK;
+  }
+  return launch_grouped_gemm_simt(A_units, B_units, C, group_offsets_dev, num_groups, total_rows, N, K, ldc,
+                                  st);
+}

@@ -1,0 +1,14 @@
+// Internal launchers behind hif4_gemm / hif4_grouped_gemm (arguments already validated).
+#pragma once
+#include "hif4_common.cuh"
+
+namespace hif4 {
+
+// CUDA-core path: any M, N, K % 64 == 0, 4-byte aligned operands.
+hif4_status launch_gemm_simt(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K,
+                             int64_t ldc, cudaStream_t st);
+hif4_status launch_grouped_gemm_simt(const void* A, const void* B, float* C, const int64_t* offsets,
+                                     int num_groups, int64_t total_rows, int64_t N, int64_t K, int64_t ldc,
+                                     cudaStream_t st);
+
+}  // namespace hif4

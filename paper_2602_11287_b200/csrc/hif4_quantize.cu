@@ -1,0 +1,386 @@
+// hif4_quantize / hif4_dequantize -- Algorithm 1 (Section II-B) and Eq. 2 of the HiFloat4 paper as
+// streaming CUDA kernels for sm_100a.  Both are bound by HBM traffic: 2 B (or 4 B) read and
+// 0.5625 B written per element for the quantizer, the reverse for the dequantizer.
+//
+// BF16 quantizer, thread mapping: 8 consecutive lanes own one 64-element unit; lane j loads the
+// 16 bytes of level-2 group j (elements 8j..8j+7) with one 128-bit load, so a warp reads 512
+// contiguous bytes (4 units) per load instruction and each lane issues kUnroll loads before it
+// computes.  Algorithm 1 is written in BF16 arithmetic; packed bf16x2 instructions with
+// round-to-nearest-even are exactly that arithmetic for two elements at a time:
+//   - peak magnitudes are integer maxima of the |x| bit patterns (NaN patterns sort above Inf);
+//   - SF = Vmax * (1/7)_BF16 is one mul.rn.bf16x2; rounding SF to the 3-bit-significand E6M2 byte is
+//     an integer add/shift on its bit pattern (the carry runs into the exponent by itself);
+//   - the E6M2 reciprocal is the 4-entry table on the mantissa plus an exponent subtraction;
+//   - rounding is monotone, so max_i bf16(|x_i| * REC) == bf16(max_i |x_i| * REC): each element is
+//     multiplied once and the micro-exponent thresholds are taken on maxima of the products;
+//   - fma.rn.bf16x2(t, 4 * 2^-(e8+e16), 128) rounds t's quarter count to nearest-even in the low
+//     mantissa bits (ulp is 1 in [128, 256)); an integer min clamps to 1.75 (and catches Inf).
+// FP32 sources run the same steps in FP32 arithmetic with 16 lanes per unit (lane = one level-3
+// group of 4 elements).
+#include <cuda_bf16.h>
+
+#include "hif4_common.cuh"
+
+namespace hif4 {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kUnroll = 4;
+
+// ----------------------------------------------------------------------------- small PTX wrappers
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t fma_bf16x2(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+// Byte permute; a selector nibble with bit 3 set replicates the selected byte's top bit.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st_stream(uint32_t* p, uint32_t v) {
+  asm volatile("st.global.cs.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void st_stream(uint4* p, uint4 v) {
+  asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
+               "r"(v.w)
+               : "memory");
+}
+__device__ __forceinline__ uint32_t umax2(uint32_t a, uint32_t b) { return __vmaxu2(a, b); }
+__device__ __forceinline__ uint32_t hmax_halves(uint32_t m) { return max(m & 0xFFFFu, m >> 16); }
+
+// E6M2 byte from the bit pattern of a non-negative, non-NaN float whose mantissa field has
+// `kMant` bits and whose exponent bias is 127: round to 2 mantissa bits, then re-bias (127 -> 48)
+// and saturate into [0x00, 0xFE].  Subnormals and everything below 2^-48 land on 0x00, Inf and
+// everything from 1.75 * 2^15 up on 0xFE.
+template <int kMant, bool kRHA>
+__device__ __forceinline__ uint32_t e6m2_from_bits(uint32_t h) {
+  constexpr int drop = kMant - 2;
+  const uint32_t half = 1u << (drop - 1);
+  const uint32_t q = kRHA ? (h + half) >> drop : (h + (half - 1) + ((h >> drop) & 1u)) >> drop;
+  const int b = static_cast<int>(q) - ((127 - 48) << 2);
+  return static_cast<uint32_t>(min(max(b, 0), 0xFE));
+}
+
+// Offset (in elements) of unit u of a [rows, upr*64] matrix with row stride ld.
+template <bool kContig>
+__device__ __forceinline__ int64_t unit_offset(int64_t u, int64_t upr, int64_t ld) {
+  if (kContig) return u * kUnitElems;
+  const int64_t r = u / upr;
+  return r * ld + (u - r * upr) * kUnitElems;
+}
+
+// ----------------------------------------------------------------------------- BF16 quantizer
+template <bool kRHA, bool kContig>
+__global__ void __launch_bounds__(kThreads)
+quantize_bf16_kernel(const uint16_t* __restrict__ src, int64_t n_units, int64_t upr, int64_t ld_src,
+                     uint32_t* __restrict__ dst) {
+  const int lane = threadIdx.x & 31;
+  const int j = lane & 7;                    // level-2 group owned by this lane
+  const int64_t warp = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) >> 5;
+  const int64_t first = warp * (4 * kUnroll) + (lane >> 3);
+
+  uint4 v[kUnroll];
+#pragma unroll
+  for (int i = 0; i < kUnroll; ++i) {
+    const int64_t u = first + 4 * i;
+    v[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (u < n_units)
+      v[i] = ld_stream(reinterpret_cast<const uint4*>(src + unit_offset<kContig>(u, upr, ld_src) + 8 * j));
+  }
+
+#pragma unroll
+  for (int i = 0; i < kUnroll; ++i) {
+    const int64_t u = first + 4 * i;
+    const uint32_t x0 = v[i].x, x1 = v[i].y, x2 = v[i].z, x3 = v[i].w;
+    const uint32_t a0 = x0 & 0x7FFF7FFFu, a1 = x1 & 0x7FFF7FFFu, a2 = x2 & 0x7FFF7FFFu,
+                   a3 = x3 & 0x7FFF7FFFu;
+    // Stage 1: peak magnitude of the unit (the group peaks are taken on the products below).
+    uint32_t vm = hmax_halves(umax2(umax2(a0, a1), umax2(a2, a3)));
+    vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 1));
+    vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 2));
+    vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 4));
+    const bool unit_nan = vm > 0x7F80u;
+
+    // Stage 2: level-1 scale, its reciprocal.
+    const uint32_t sf = mul_bf16x2(vm, 0x3E12u) & 0xFFFFu;             // Vmax * (1/7)_BF16
+    const uint32_t byte = e6m2_from_bits<7, kRHA>(sf);
+    const uint32_t lut = (0x122B4D80u >> ((byte & 3u) * 8u)) & 0xFFu;   // 1/1.M in BF16: 3F80 3F4D 3F2B 3F12
+    const uint32_t rec = (0x3F00u | lut) + (48u << 7) - ((byte >> 2) << 7);
+    const uint32_t rec2 = rec * 0x10001u;
+
+    const uint32_t t0 = mul_bf16x2(a0, rec2), t1 = mul_bf16x2(a1, rec2), t2 = mul_bf16x2(a2, rec2),
+                   t3 = mul_bf16x2(a3, rec2);
+    // Level-2 and level-3 micro-exponents from the peaks of the products.
+    const uint32_t p16a = hmax_halves(umax2(t0, t1));     // elements 0..3 of this lane
+    const uint32_t p16b = hmax_halves(umax2(t2, t3));     // elements 4..7
+    const uint32_t e8 = max(p16a, p16b) >= 0x4080u;       // >= 4.0
+    const uint32_t thr = 0x4000u + (e8 << 7);             // 2.0 * 2^e8
+    const uint32_t e16a = p16a >= thr, e16b = p16b >= thr;
+
+    // Stage 3: quarter counts 4 * t * 2^-(e8+e16), rounded, clamped to 7.
+    uint32_t c0, c1, c2, c3;
+    if (!kRHA) {
+      const uint32_t mula = (0x4080u - ((e8 + e16a) << 7)) * 0x10001u;
+      const uint32_t mulb = (0x4080u - ((e8 + e16b) << 7)) * 0x10001u;
+      c0 = __vminu2(fma_bf16x2(t0, mula, 0x43004300u), 0x43074307u);
+      c1 = __vminu2(fma_bf16x2(t1, mula, 0x43004300u), 0x43074307u);
+      c2 = __vminu2(fma_bf16x2(t2, mulb, 0x43004300u), 0x43074307u);
+      c3 = __vminu2(fma_bf16x2(t3, mulb, 0x43004300u), 0x43074307u);
+    } else {
+      // round-half-away: widen to FP32 (exact), add one half, truncate
+      const float fa = __uint_as_float((129u - (e8 + e16a)) << 23);
+      const float fb = __uint_as_float((129u - (e8 + e16b)) << 23);
+      auto rha = [](uint32_t t, float f) {
+        const float lo = fminf(__uint_as_float(t << 16) * f, 8.0f);
+        const float hi = fminf(__uint_as_float(t & 0xFFFF0000u) * f, 8.0f);
+        const uint32_t ql = min(static_cast<uint32_t>(lo + 0.5f), 7u);
+        const uint32_t qh = min(static_cast<uint32_t>(hi + 0.5f), 7u);
+        return 0x43004300u | ql | (qh << 16);
+      };
+      c0 = rha(t0, fa); c1 = rha(t1, fa); c2 = rha(t2, fb); c3 = rha(t3, fb);
+    }
+    // Pack: low bytes of the four bf16x2 results hold the magnitudes; signs come from the top bit of
+    // each source element.  Pairs are gathered in swapped order so that one multiply by 0x1001
+    // drops (q_even | q_odd << 4) into bytes 1 and 3.
+    uint32_t g0 = prmt(c0, c1, 0x4602u), g1 = prmt(c2, c3, 0x4602u);
+    g0 |= prmt(x0, x1, 0xDF9Bu) & 0x08080808u;
+    g1 |= prmt(x2, x3, 0xDF9Bu) & 0x08080808u;
+    uint32_t codes = prmt(g0 * 0x1001u, g1 * 0x1001u, 0x7531u);
+
+    uint32_t meta = (e8 << (8 + j)) | (e16a << (16 + 2 * j)) | (e16b << (17 + 2 * j));
+    meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 1);
+    meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 2);
+    meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 4);
+    meta |= byte;
+    if (unit_nan) { meta = 0xFFu; codes = 0u; }          // NaN unit: E6M2 = NaN, everything else zero
+
+    if (u < n_units) {
+      uint32_t* out = dst + u * kUnitWords;
+      st_stream(out + 1 + j, codes);
+      if (j == 0) st_stream(out, meta);
+    }
+  }
+}
+
+// ----------------------------------------------------------------------------- FP32 quantizer
+// 16 lanes per unit, lane k owns level-3 group k (elements 4k..4k+3); lanes 2j, 2j+1 form level-2
+// group j.  Same steps as above in FP32 arithmetic: (1/7) and the reciprocal table are the nearest
+// FP32 values, every product is a single mul.rn.f32.
+template <bool kRHA, bool kContig>
+__global__ void __launch_bounds__(kThreads)
+quantize_fp32_kernel(const float* __restrict__ src, int64_t n_units, int64_t upr, int64_t ld_src,
+                     uint32_t* __restrict__ dst) {
+  const int lane = threadIdx.x & 31;
+  const int k = lane & 15;
+  const int64_t warp = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) >> 5;
+  const int64_t first = warp * (2 * kUnroll) + (lane >> 4);
+
+  uint4 v[kUnroll];
+#pragma unroll
+  for (int i = 0; i < kUnroll; ++i) {
+    const int64_t u = first + 2 * i;
+    v[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (u < n_units)
+      v[i] = ld_stream(reinterpret_cast<const uint4*>(src + unit_offset<kContig>(u, upr, ld_src) + 4 * k));
+  }
+
+#pragma unroll
+  for (int i = 0; i < kUnroll; ++i) {
+    const int64_t u = first + 2 * i;
+    const uint32_t xb[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+    uint32_t ab[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) ab[e] = xb[e] & 0x7FFFFFFFu;
+    uint32_t vm = max(max(ab[0], ab[1]), max(ab[2], ab[3]));
+#pragma unroll
+    for (int s = 1; s < 16; s <<= 1) vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, s));
+    const bool unit_nan = vm > 0x7F800000u;
+
+    const float sf = __fmul_rn(__uint_as_float(vm), __uint_as_float(0x3E124925u));   // (1/7)_FP32
+    const uint32_t byte = e6m2_from_bits<23, kRHA>(__float_as_uint(sf));
+    const uint32_t M = byte & 3u;
+    // nearest FP32 of 1, 0.8, 2/3, 4/7
+    const uint32_t lut = M == 0 ? 0x3F800000u : M == 1 ? 0x3F4CCCCDu : M == 2 ? 0x3F2AAAABu : 0x3F124925u;
+    const float rec = __uint_as_float(lut + (48u << 23) - ((byte >> 2) << 23));
+
+    float t[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) t[e] = __fmul_rn(__uint_as_float(ab[e]), rec);
+    const uint32_t p16 = max(max(__float_as_uint(t[0]), __float_as_uint(t[1])),
+                             max(__float_as_uint(t[2]), __float_as_uint(t[3])));
+    const uint32_t p8 = max(p16, __shfl_xor_sync(0xFFFFFFFFu, p16, 1));
+    const uint32_t e8 = p8 >= 0x40800000u;                     // >= 4.0
+    const uint32_t e16 = p16 >= 0x40000000u + (e8 << 23);      // >= 2.0 * 2^e8
+    const float mul = __uint_as_float((129u - (e8 + e16)) << 23);   // 4 * 2^-(e8+e16)
+
+    uint32_t half = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float q = fminf(__fmul_rn(t[e], mul), 8.0f);
+      uint32_t m;
+      if (!kRHA) {
+        m = static_cast<uint32_t>(__float2int_rn(q));
+      } else {
+        const float fl = truncf(q);
+        m = static_cast<uint32_t>(fl) + ((q - fl) >= 0.5f ? 1u : 0u);
+      }
+      m = min(m, 7u) | ((xb[e] >> 28) & 8u);
+      half |= m << (4 * e);
+    }
+    const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, half, 1);
+    uint32_t codes = half | (other << 16);                      // meaningful on even lanes
+
+    uint32_t meta = (e16 << (16 + k)) | ((k & 1) ? 0u : (e8 << (8 + (k >> 1))));
+#pragma unroll
+    for (int s = 1; s < 16; s <<= 1) meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, s);
+    meta |= byte;
+    if (unit_nan) { meta = 0xFFu; codes = 0u; }
+
+    if (u < n_units) {
+      uint32_t* out = dst + u * kUnitWords;
+      if ((k & 1) == 0) st_stream(out + 1 + (k >> 1), codes);
+      if (k == 0) st_stream(out, meta);
+    }
+  }
+}
+
+// ----------------------------------------------------------------------------- dequantizer (Eq. 2)
+// 8 lanes per unit; lane j decodes code word j (elements 8j..8j+7).  Each value is
+// m * (4+M) * 2^(E-48-4+e8+e16): an integer below 64 times a power of two, exact in FP32 and BF16.
+template <bool kBF16Out, bool kContig>
+__global__ void __launch_bounds__(kThreads)
+dequantize_kernel(const uint32_t* __restrict__ src, int64_t n_units, int64_t upr, int64_t ld_dst,
+                  void* __restrict__ dst) {
+  const int lane = threadIdx.x & 31;
+  const int j = lane & 7;
+  const int64_t warp = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) >> 5;
+  const int64_t first = warp * (4 * kUnroll) + (lane >> 3);
+
+  uint32_t meta[kUnroll], word[kUnroll];
+#pragma unroll
+  for (int i = 0; i < kUnroll; ++i) {
+    const int64_t u = first + 4 * i;
+    meta[i] = 0; word[i] = 0;
+    if (u < n_units) {
+      meta[i] = __ldg(src + u * kUnitWords);
+      word[i] = __ldg(src + u * kUnitWords + 1 + j);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kUnroll; ++i) {
+    const int64_t u = first + 4 * i;
+    if (u >= n_units) continue;
+    const uint32_t byte = meta[i] & 0xFFu;
+    const uint32_t e8 = (meta[i] >> (8 + j)) & 1u;
+    const uint32_t e16a = (meta[i] >> (16 + 2 * j)) & 1u, e16b = (meta[i] >> (17 + 2 * j)) & 1u;
+    const float mant = static_cast<float>(4u + (byte & 3u));
+    // exponent field of 2^(E - 48 - 4 + shift): (byte >> 2) - 52 + 127 + shift
+    const float sa = mant * __uint_as_float(((byte >> 2) + 75u + e8 + e16a) << 23);
+    const float sb = mant * __uint_as_float(((byte >> 2) + 75u + e8 + e16b) << 23);
+    uint32_t bits[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const uint32_t c = (word[i] >> (4 * e)) & 0xFu;
+      const float val = static_cast<float>(c & 7u) * (e < 4 ? sa : sb);
+      bits[e] = byte == 0xFFu ? 0x7FC00000u : (__float_as_uint(val) | ((c & 8u) << 28));
+    }
+    const int64_t off = unit_offset<kContig>(u, upr, ld_dst) + 8 * j;
+    if (kBF16Out) {
+      uint4 o;
+      o.x = (bits[0] >> 16) | (bits[1] & 0xFFFF0000u);
+      o.y = (bits[2] >> 16) | (bits[3] & 0xFFFF0000u);
+      o.z = (bits[4] >> 16) | (bits[5] & 0xFFFF0000u);
+      o.w = (bits[6] >> 16) | (bits[7] & 0xFFFF0000u);
+      st_stream(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + off), o);
+    } else {
+      uint4* p = reinterpret_cast<uint4*>(static_cast<float*>(dst) + off);
+      st_stream(p, make_uint4(bits[0], bits[1], bits[2], bits[3]));
+      st_stream(p + 1, make_uint4(bits[4], bits[5], bits[6], bits[7]));
+    }
+  }
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+}  // namespace
+}  // namespace hif4
+
+using namespace hif4;
+
+extern "C" hif4_status hif4_quantize(const void* src, hif4_dtype dt, int64_t rows, int64_t cols,
+                                     int64_t ld_src, void* dst_units, hif4_round mode, void* stream) {
+  if (dt != HIF4_BF16 && dt != HIF4_FP32) return HIF4_ERR_DTYPE;
+  if (mode != HIF4_RNE && mode != HIF4_RHA) return HIF4_ERR_DTYPE;
+  if (rows < 0 || cols < 0 || cols % kUnitElems != 0 || ld_src < cols) return HIF4_ERR_SHAPE;
+  if (rows == 0 || cols == 0) return HIF4_OK;
+  if (!src || !dst_units) return HIF4_ERR_NULL;
+  const size_t esz = dt == HIF4_BF16 ? 2 : 4;
+  if (!aligned(src, 16) || (static_cast<size_t>(ld_src) * esz) % 16 != 0 || !aligned(dst_units, 4))
+    return HIF4_ERR_ALIGN;
+  const int64_t upr = cols / kUnitElems;
+  const int64_t n_units = rows * upr;
+  const bool contig = ld_src == cols;
+  const int units_per_block = (kThreads / 32) * kUnroll * (dt == HIF4_BF16 ? 4 : 2);
+  const int64_t blocks = ceil_div64(n_units, units_per_block);
+  if (blocks > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t* dst = static_cast<uint32_t*>(dst_units);
+  const dim3 grid(static_cast<unsigned>(blocks));
+#define HIF4_LAUNCH_Q(KERNEL, T)                                                                 \
+  do {                                                                                           \
+    if (mode == HIF4_RNE) {                                                                      \
+      if (contig) KERNEL<false, true><<<grid, kThreads, 0, st>>>(static_cast<const T*>(src), n_units, upr, ld_src, dst); \
+      else KERNEL<false, false><<<grid, kThreads, 0, st>>>(static_cast<const T*>(src), n_units, upr, ld_src, dst);       \
+    } else {                                                                                     \
+      if (contig) KERNEL<true, true><<<grid, kThreads, 0, st>>>(static_cast<const T*>(src), n_units, upr, ld_src, dst);  \
+      else KERNEL<true, false><<<grid, kThreads, 0, st>>>(static_cast<const T*>(src), n_units, upr, ld_src, dst);        \
+    }                                                                                            \
+  } while (0)
+  if (dt == HIF4_BF16) HIF4_LAUNCH_Q(quantize_bf16_kernel, uint16_t);
+  else HIF4_LAUNCH_Q(quantize_fp32_kernel, float);
+#undef HIF4_LAUNCH_Q
+  note_launch();
+  return launch_status();
+}
+
+extern "C" hif4_status hif4_dequantize(const void* src_units, int64_t rows, int64_t cols, void* dst,
+                                       hif4_dtype dt, int64_t ld_dst, void* stream) {
+  if (dt != HIF4_BF16 && dt != HIF4_FP32) return HIF4_ERR_DTYPE;
+  if (rows < 0 || cols < 0 || cols % kUnitElems != 0 || ld_dst < cols) return HIF4_ERR_SHAPE;
+  if (rows == 0 || cols == 0) return HIF4_OK;
+  if (!src_units || !dst) return HIF4_ERR_NULL;
+  const size_t esz = dt == HIF4_BF16 ? 2 : 4;
+  if (!aligned(dst, 16) || (static_cast<size_t>(ld_dst) * esz) % 16 != 0 || !aligned(src_units, 4))
+    return HIF4_ERR_ALIGN;
+  const int64_t upr = cols / kUnitElems;
+  const int64_t n_units = rows * upr;
+  const bool contig = ld_dst == cols;
+  const int64_t blocks = ceil_div64(n_units, (kThreads / 32) * kUnroll * 4);
+  if (blocks > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const uint32_t* in = static_cast<const uint32_t*>(src_units);
+  const dim3 grid(static_cast<unsigned>(blocks));
+  if (dt == HIF4_BF16) {
+    if (contig) dequantize_kernel<true, true><<<grid, kThreads, 0, st>>>(in, n_units, upr, ld_dst, dst);
+    else dequantize_kernel<true, false><<<grid, kThreads, 0, st>>>(in, n_units, upr, ld_dst, dst);
+  } else {
+    if (contig) dequantize_kernel<false, true><<<grid, kThreads, 0, st>>>(in, n_units, upr, ld_dst, dst);
+    else dequantize_kernel<false, false><<<grid, kThreads, 0, st>>>(in, n_units, upr, ld_dst, dst);
+  }
+  note_launch();
+  return launch_status();
+}

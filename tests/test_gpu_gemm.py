@@ -1,0 +1,143 @@
+"""GPU parity for hif4_gemm / hif4_grouped_gemm through the C ABI:
+max |C_gpu - C_ref| <= 1e-5 * sum_k |a_ik| |b_jk| against the FP64 oracle on the decoded operands."""
+import numpy as np
+import pytest
+import torch
+
+import hif4_workloads as wl
+import oracle
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def hif4():
+    assert torch.cuda.is_available()
+    import paper_2602_11287_b200 as lib
+    return lib
+
+
+def check_full(hif4, a_units, b_units, what, out=None):
+    C = hif4.hif4_gemm(a_units, b_units, out=out)
+    ref, refabs = oracle.gemm_f64(a_units.cpu().numpy(), b_units.cpu().numpy(), nthreads=8)
+    got = C.cpu().numpy().astype(np.float64)
+    err = np.abs(got - ref)
+    bound = TOL * refabs
+    assert np.all(err <= bound + 1e-300), f"{what}: worst ratio {np.max(err / np.maximum(bound, 1e-300)):.3g}"
+    return C
+
+
+def check_sampled(hif4, a_units, b_units, what, n=600, seed=0, C=None):
+    if C is None:
+        C = hif4.hif4_gemm(a_units, b_units)
+    M, N = C.shape
+    rng = np.random.default_rng(seed)
+    rows = np.concatenate([rng.integers(0, M, n), [0, M - 1, 0, M - 1]])
+    cols = np.concatenate([rng.integers(0, N, n), [0, 0, N - 1, N - 1]])
+    ref, refabs = oracle.gemm_sampled_f64(a_units.cpu().numpy(), b_units.cpu().numpy(), rows, cols)
+    got = C[torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()].cpu().numpy().astype(np.float64)
+    err = np.abs(got - ref)
+    assert np.all(err <= TOL * refabs + 1e-300), f"{what}: worst ratio {np.max(err / np.maximum(TOL * refabs, 1e-300)):.3g}"
+    return C
+
+
+def test_single_layer_config(hif4):
+    x, w = wl.single_layer(device="cuda")
+    check_full(hif4, hif4.hif4_quantize(x), hif4.hif4_quantize(w), "cfg1 128x512x512")
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 64, 64), (1, 1, 64), (3, 5, 128), (64, 64, 64), (65, 63, 192), (130, 257, 320),
+                                   (16, 200, 1024), (200, 16, 256), (129, 300, 768), (257, 513, 256)])
+def test_small_and_ragged_shapes(hif4, M, N, K):
+    g = torch.Generator(device="cuda"); g.manual_seed(M * 1000 + N)
+    a = torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16)
+    b = (torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16)
+    check_full(hif4, hif4.hif4_quantize(a), hif4.hif4_quantize(b), f"{M}x{N}x{K}")
+
+
+def test_random_units_all_scales_and_strided_c(hif4):
+    rng = np.random.default_rng(21)
+    M, N, upr = 70, 90, 4
+    A = rng.integers(0, 256, (M, upr, 36), dtype=np.uint8)
+    B = rng.integers(0, 256, (N, upr, 36), dtype=np.uint8)
+    A[..., 0] = rng.integers(0x60, 0xE0, (M, upr)); B[..., 0] = rng.integers(0x60, 0xE0, (N, upr))
+    out = torch.full((M, 96), -5.0, dtype=torch.float32, device="cuda")
+    check_full(hif4, torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), "random units", out=out[:, :N])
+    assert (out[:, N:] == -5.0).all()
+
+
+def test_nan_units_and_determinism(hif4):
+    rng = np.random.default_rng(22)
+    A = rng.integers(0, 256, (66, 4, 36), dtype=np.uint8); A[..., 0] = 0xC0
+    B = rng.integers(0, 256, (70, 4, 36), dtype=np.uint8); B[..., 0] = 0xB0
+    A[5, 2, 0] = 0xFF
+    B[69, 0, 0] = 0xFF
+    a, b = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+    C = hif4.hif4_gemm(a, b)
+    nan = torch.isnan(C).cpu().numpy()
+    want = np.zeros((66, 70), bool); want[5, :] = True; want[:, 69] = True
+    assert np.array_equal(nan, want)
+    C2 = hif4.hif4_gemm(a, b)
+    assert torch.equal(torch.nan_to_num(C), torch.nan_to_num(C2)), "two runs differ"
+
+
+def test_llama_shapes_sampled(hif4):
+    for (name, K, N) in wl.LLAMA3_8B_LINEARS:
+        w = hif4.hif4_quantize(wl.gaussian(N, K, 0.02, seed=2000 + N + K, device="cuda"))
+        for M in (1, 16, 512):
+            x = hif4.hif4_quantize(wl.llama_activations(M, K, device="cuda"))
+            check_sampled(hif4, x, w, f"llama {name} M={M}", n=300)
+
+
+def test_empty_and_bad_arguments(hif4):
+    a = torch.zeros(0, 2, 36, dtype=torch.uint8, device="cuda")
+    b = torch.zeros(5, 2, 36, dtype=torch.uint8, device="cuda")
+    assert hif4.hif4_gemm(a, b).shape == (0, 5)
+    a = torch.zeros(3, 0, 36, dtype=torch.uint8, device="cuda")
+    b = torch.zeros(5, 0, 36, dtype=torch.uint8, device="cuda")
+    out = torch.ones(3, 8, dtype=torch.float32, device="cuda")
+    hif4.hif4_gemm(a, b, out=out[:, :5])          # K == 0: zero fill of the [M, N] window only
+    assert (out[:, :5] == 0).all() and (out[:, 5:] == 1).all()
+    import ctypes
+    n = ctypes.c_size_t(0)
+    assert hif4.lib.hif4_gemm_workspace(4, 4, 100, ctypes.byref(n)) == 2
+    assert hif4.lib.hif4_gemm(None, None, None, 4, 4, 64, 4, None, 0, None) == 1
+    c = torch.zeros(4, 6, dtype=torch.float32, device="cuda")
+    au = torch.zeros(4, 1, 36, dtype=torch.uint8, device="cuda")
+    assert hif4.lib.hif4_gemm(au.data_ptr() + 2, au.data_ptr(), c.data_ptr(), 4, 4, 64, 6, None, 0, None) == 3   # A % 4
+    assert hif4.lib.hif4_gemm(au.data_ptr(), au.data_ptr(), c.data_ptr(), 4, 4, 64, 2, None, 0, None) == 2   # ldc < N
+
+
+def _grouped_case(hif4, counts, N, K, seed):
+    g = torch.Generator(device="cuda"); g.manual_seed(seed)
+    G = len(counts)
+    off = torch.zeros(G + 1, dtype=torch.int64)
+    off[1:] = torch.cumsum(torch.tensor(counts), 0)
+    total = int(off[-1])
+    a = hif4.hif4_quantize(torch.randn(max(total, 1), K, generator=g, device="cuda").to(torch.bfloat16))[:total]
+    b = hif4.hif4_quantize((torch.randn(G * N, K, generator=g, device="cuda") * 0.02).to(torch.bfloat16)).view(G, N, K // 64, 36)
+    out = torch.full((total, N), 3.0, dtype=torch.float32, device="cuda")
+    hif4.hif4_grouped_gemm(a, b, off.cuda(), out=out)
+    ref, refabs = oracle.grouped_gemm_f64(a.cpu().numpy(), b.cpu().numpy(), off.numpy(), nthreads=8)
+    err = np.abs(out.cpu().numpy().astype(np.float64) - ref)
+    assert np.all(err <= TOL * refabs + 1e-300)
+
+
+def test_grouped_gemm_with_empty_and_ragged_groups(hif4):
+    _grouped_case(hif4, [3, 0, 70, 1, 0, 129, 64, 0], N=96, K=256, seed=31)
+    _grouped_case(hif4, [0, 0, 5], N=64, K=64, seed=32)
+    _grouped_case(hif4, [200], N=130, K=512, seed=33)
+
+
+def test_grouped_gemm_moe_routing_sampled(hif4):
+    r = wl.moe_routing(tokens=512, experts=32, topk=4, device="cuda")
+    off = r["offsets"]
+    total = int(off[-1])
+    K, N, G = 512, 256, 32
+    a = hif4.hif4_quantize(wl.outlier_channel_activations(total, K, seed=41, device="cuda"))
+    b = hif4.hif4_quantize(wl.gaussian(G * N, K, 0.02, seed=42, device="cuda")).view(G, N, K // 64, 36)
+    out = hif4.hif4_grouped_gemm(a, b, off)
+    ref, refabs = oracle.grouped_gemm_f64(a.cpu().numpy(), b.cpu().numpy(), off.cpu().numpy(), nthreads=8)
+    err = np.abs(out.cpu().numpy().astype(np.float64) - ref)
+    assert np.all(err <= TOL * refabs + 1e-300)

@@ -1,0 +1,146 @@
+"""GPU parity, bit-exact: hif4_quantize / hif4_dequantize through the C ABI against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import hif4_workloads as wl
+import oracle
+from tests import adversarial
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def hif4():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    import paper_2602_11287_b200 as lib
+    return lib
+
+
+def _gpu_quantize_bits(hif4, bits_u16, mode=0):
+    t = wl.u16_numpy_to_bf16(bits_u16, "cuda")
+    return hif4.hif4_quantize(t, mode).cpu().numpy()
+
+
+def _compare_units(got, want, what):
+    if np.array_equal(got, want):
+        return
+    bad = np.argwhere((got != want).any(axis=-1))
+    r, u = bad[0]
+    raise AssertionError(f"{what}: {len(bad)} of {got.shape[0] * got.shape[1]} units differ; first at row {r} unit {u}: "
+                         f"gpu {got[r, u].tobytes().hex()} oracle {want[r, u].tobytes().hex()}")
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_quantize_bf16_every_magnitude_under_many_peaks(hif4, mode):
+    peaks = [0x4000 | m for m in range(0, 128, 3)] + [0x3F80, 0x3FFF, 0x40E0, 0x4100]
+    bits = adversarial.bf16_sweep_units(peaks, 0x0000, 0x4200, seed=mode)
+    got = _gpu_quantize_bits(hif4, bits, mode)
+    want = oracle.quantize(bits, mode, nthreads=8)
+    _compare_units(got, want, f"bf16 sweep mode {mode}")
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_quantize_bf16_specials_and_extremes(hif4, mode):
+    bits = adversarial.bf16_special_units()
+    got = _gpu_quantize_bits(hif4, bits, mode)
+    want = oracle.quantize(bits, mode)
+    _compare_units(got, want, "bf16 specials")
+    # whole-range sweep with huge / tiny peaks
+    bits = adversarial.bf16_sweep_units([0x7F7F, 0x7F80, 0x4780, 0x2A00, 0x0100, 0x0040], 0, 0x7F80, seed=3)
+    _compare_units(_gpu_quantize_bits(hif4, bits, mode), oracle.quantize(bits, mode, nthreads=8), "bf16 extremes")
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_quantize_fp32_adversarial(hif4, mode):
+    x = adversarial.fp32_adversarial(seed=mode)
+    got = hif4.hif4_quantize(torch.from_numpy(x).cuda(), mode).cpu().numpy()
+    want = oracle.quantize(x, mode, nthreads=8)
+    _compare_units(got, want, f"fp32 adversarial mode {mode}")
+
+
+def test_quantize_workload_distributions(hif4):
+    x, w = wl.single_layer(device="cuda")
+    for t in (x, w):
+        _compare_units(hif4.hif4_quantize(t).cpu().numpy(), oracle.quantize(wl.bf16_to_u16_numpy(t), nthreads=8), "cfg1")
+    t = wl.llama_activations(48, 4096, device="cuda")
+    _compare_units(hif4.hif4_quantize(t).cpu().numpy(), oracle.quantize(wl.bf16_to_u16_numpy(t), nthreads=8), "cfg2")
+    t = wl.quantize_sweep(2 ** 20, device="cuda")
+    _compare_units(hif4.hif4_quantize(t).cpu().numpy(), oracle.quantize(wl.bf16_to_u16_numpy(t), nthreads=8), "cfg3")
+    t32 = wl.quantize_sweep(2 ** 18, device="cuda", dtype=torch.float32)
+    _compare_units(hif4.hif4_quantize(t32).cpu().numpy(), oracle.quantize(t32.cpu().numpy(), nthreads=8), "cfg3 fp32")
+    t = wl.prefill_activations(64, 5120, device="cuda")
+    _compare_units(hif4.hif4_quantize(t).cpu().numpy(), oracle.quantize(wl.bf16_to_u16_numpy(t), nthreads=8), "cfg4")
+
+
+def test_quantize_ragged_sizes_strided_rows_and_guard_bands(hif4):
+    g = torch.Generator(device="cuda"); g.manual_seed(5)
+    for rows, cols, ld in [(1, 64, 64), (3, 64, 72), (5, 192, 192), (7, 320, 384), (33, 448, 448), (130, 64, 64),
+                           (1, 4096, 4096), (17, 1088, 1096)]:
+        for dtype in (torch.bfloat16, torch.float32):
+            buf = torch.randn(rows, ld, generator=g, device="cuda", dtype=torch.float32).to(dtype)
+            src = buf[:, :cols]
+            upr = cols // 64
+            out = torch.full((rows * upr * 36 + 128,), 0xAB, dtype=torch.uint8, device="cuda")
+            view = out[64:64 + rows * upr * 36].view(rows, upr, 36)
+            hif4.hif4_quantize(src, out=view)
+            host = src.contiguous().cpu()
+            ref = oracle.quantize(wl.bf16_to_u16_numpy(host) if dtype == torch.bfloat16 else host.numpy())
+            _compare_units(view.cpu().numpy(), ref, f"ragged {rows}x{cols} ld {ld} {dtype}")
+            o = out.cpu().numpy()
+            assert (o[:64] == 0xAB).all() and (o[64 + rows * upr * 36:] == 0xAB).all(), "guard band overwritten"
+
+
+def test_quantize_empty_and_bad_arguments(hif4):
+    e = torch.empty(0, 128, dtype=torch.bfloat16, device="cuda")
+    assert hif4.hif4_quantize(e).shape == (0, 2, 36)
+    x = torch.zeros(4, 100, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(hif4.Hif4Error) as ei:
+        hif4.hif4_quantize(x, out=torch.empty(4, 1, 36, dtype=torch.uint8, device="cuda"))
+    assert ei.value.code == 2
+    x = torch.zeros(4, 136, dtype=torch.bfloat16, device="cuda")[:, 4:132]     # rows not 16-byte aligned
+    with pytest.raises(hif4.Hif4Error) as ei:
+        hif4.hif4_quantize(x)
+    assert ei.value.code == 3
+    with pytest.raises(hif4.Hif4Error) as ei:
+        hif4.hif4_quantize(torch.zeros(2, 64, dtype=torch.bfloat16, device="cuda"), mode=7)
+    assert ei.value.code == 4
+    with pytest.raises(TypeError):
+        hif4.hif4_quantize(torch.zeros(2, 64, dtype=torch.float16, device="cuda"))
+    with pytest.raises(ValueError):
+        hif4.hif4_quantize(torch.zeros(2, 64, dtype=torch.bfloat16))
+    assert hif4.hif4_last_device_status() == 0
+
+
+def test_dequantize_every_code_and_metadata_value(hif4):
+    rng = np.random.default_rng(6)
+    # all 256 level-1 bytes (incl. NaN) x random micro-exponents and codes, plus fully random units
+    u = rng.integers(0, 256, size=(256 * 8, 3, 36), dtype=np.uint8)
+    u[:, :, 0] = (np.arange(256 * 8) % 256)[:, None]
+    # make sure every (e8, e16, code) combination occurs under every byte: structured units
+    s = np.zeros((256, 4, 36), dtype=np.uint8)
+    for b in range(256):
+        for v, (e8, e16) in enumerate([(0, 0), (0, 0xFFFF), (0xFF, 0), (0xFF, 0xFFFF)]):
+            s[b, v, 0] = b; s[b, v, 1] = e8; s[b, v, 2] = e16 & 0xFF; s[b, v, 3] = e16 >> 8
+            s[b, v, 4:] = np.tile(np.array([0x10, 0x32, 0x54, 0x76, 0x98, 0xBA, 0xDC, 0xFE], dtype=np.uint8), 4)
+    for units in (u, s):
+        dev = torch.from_numpy(units).cuda()
+        got16 = hif4.hif4_dequantize(dev, torch.bfloat16)
+        got32 = hif4.hif4_dequantize(dev, torch.float32)
+        want16 = oracle.dequantize(units, oracle.BF16)
+        want32 = oracle.dequantize(units, oracle.FP32)
+        assert np.array_equal(wl.bf16_to_u16_numpy(got16), want16)
+        assert np.array_equal(got32.cpu().numpy().view(np.uint32), want32.view(np.uint32))
+
+
+def test_dequantize_strided_output_and_roundtrip(hif4):
+    t = wl.llama_activations(19, 1088, device="cuda")
+    units = hif4.hif4_quantize(t)
+    buf = torch.full((19, 1100), 7.0, dtype=torch.float32, device="cuda")
+    hif4.hif4_dequantize(units, out=buf[:, :1088])
+    ref = oracle.dequantize(oracle.quantize(wl.bf16_to_u16_numpy(t)), oracle.FP32)
+    assert np.array_equal(buf[:, :1088].cpu().numpy().view(np.uint32), ref.view(np.uint32))
+    assert (buf[:, 1088:] == 7.0).all()
+    # the "simulated 4-bit" tensor stays close to the source (3-bit significand, shared scales)
+    rel = (buf[:, :1088] - t.float()).norm() / t.float().norm()
+    assert rel < 0.15
