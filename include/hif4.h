@@ -131,6 +131,11 @@ hif4_status hif4_last_device_status(void* stream);
 /* Static, NUL-terminated description of a status code.  Host-only.  */
 const char* hif4_status_string(hif4_status s);
 
+/* Diagnostic: 0 = choose the GEMM kernel by shape (default), 1 = CUDA-core kernel only, 2 = the
+ * tensor-core (tcgen05) kernel whenever it is legal (K % 256 == 0, 16-byte aligned operands), even
+ * for small M.  Process-wide, not thread-safe; meant for tests and benchmarks.  */
+hif4_status hif4_set_gemm_path(int path);
+
 /* Number of kernels this library has launched in this process (monotonic, host-side counter).  */
 uint64_t hif4_launch_count(void);
 

@@ -23,7 +23,7 @@ HIF4_OK = 0
 EXPORTED_SYMBOLS = [
     "hif4_packed_bytes", "hif4_quantize", "hif4_dequantize", "hif4_gemm_workspace", "hif4_gemm",
     "hif4_grouped_gemm_workspace", "hif4_grouped_gemm", "hif4_last_device_status", "hif4_status_string",
-    "hif4_launch_count",
+    "hif4_launch_count", "hif4_set_gemm_path",
 ]
 
 
@@ -58,6 +58,8 @@ def _load() -> ctypes.CDLL:
     L.hif4_last_device_status.argtypes = [vp]
     L.hif4_status_string.restype = ctypes.c_char_p
     L.hif4_status_string.argtypes = [ci]
+    L.hif4_set_gemm_path.restype = ci
+    L.hif4_set_gemm_path.argtypes = [ci]
     L.hif4_launch_count.restype = ctypes.c_uint64
     L.hif4_launch_count.argtypes = []
     return L
@@ -194,6 +196,11 @@ def hif4_grouped_gemm(a_units: torch.Tensor, b_units: torch.Tensor, group_offset
                                  G, total, N, K, ldc, workspace.data_ptr() if workspace is not None else None,
                                  workspace.numel() if workspace is not None else 0, _stream(stream)))
     return out
+
+
+def hif4_set_gemm_path(path: int) -> None:
+    """0 = by shape, 1 = CUDA-core kernel only, 2 = tensor-core kernel whenever legal."""
+    _check("hif4_set_gemm_path", lib.hif4_set_gemm_path(path))
 
 
 def hif4_last_device_status(stream=None) -> int:

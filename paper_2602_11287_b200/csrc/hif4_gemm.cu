@@ -5,6 +5,10 @@
 using namespace hif4;
 
 namespace {
+// 0 = choose by shape, 1 = CUDA-core kernel only, 2 = tensor-core kernel whenever it is legal.
+int g_gemm_path = 0;
+constexpr int64_t kTensorCoreMinM = 64;
+
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 hif4_status check_common(const void* A, const void* B, const float* C, int64_t M, int64_t N, int64_t K,
@@ -24,6 +28,12 @@ extern "C" hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size
   return HIF4_OK;
 }
 
+extern "C" hif4_status hif4_set_gemm_path(int path) {
+  if (path < 0 || path > 2) return HIF4_ERR_DTYPE;
+  g_gemm_path = path;
+  return HIF4_OK;
+}
+
 extern "C" hif4_status hif4_gemm(const void* A_units, const void* B_units, float* C, int64_t M, int64_t N,
                                  int64_t K, int64_t ldc, void* workspace, size_t workspace_bytes,
                                  void* stream) {
@@ -38,6 +48,8 @@ extern "C" hif4_status hif4_gemm(const void* A_units, const void* B_units, float
       return HIF4_ERR_CUDA;
     return HIF4_OK;
   }
+  const bool tc_ok = g_gemm_path != 1 && gemm_tc_supported(A_units, B_units, M, N, N, K);
+  if (tc_ok && (g_gemm_path == 2 || M >= kTensorCoreMinM)) return launch_gemm_tc(A_units, B_units, C, M, N, K, ldc, st);
   return launch_gemm_simt(A_units, B_units, C, M, N, K, ldc, st);
 }
 
@@ -45,7 +57,8 @@ extern "C" hif4_status hif4_grouped_gemm_workspace(int num_groups, int64_t total
                                                    size_t* bytes) {
   if (!bytes) return HIF4_ERR_NULL;
   if (num_groups < 0 || total_rows < 0 || N < 0 || K < 0 || K % kUnitElems != 0) return HIF4_ERR_SHAPE;
-  *bytes = 0;
+  // the tensor-core path keeps its tile table (one 16-byte entry per 128-row tile) here
+  *bytes = (K > 0 && K % 256 == 0 && total_rows > 0 && num_groups > 0) ? grouped_tc_workspace_bytes(num_groups, total_rows) : 0;
   return HIF4_OK;
 }
 
@@ -53,8 +66,6 @@ extern "C" hif4_status hif4_grouped_gemm(const void* A_units, const void* B_unit
                                          const int64_t* group_offsets_dev, int num_groups, int64_t total_rows,
                                          int64_t N, int64_t K, int64_t ldc, void* workspace,
                                          size_t workspace_bytes, void* stream) {
-  (void)workspace;
-  (void)workspace_bytes;
   if (num_groups < 0) return HIF4_ERR_SHAPE;
   const hif4_status chk = check_common(A_units, B_units, C, total_rows, N, K, ldc);
   if (chk != HIF4_OK || total_rows == 0 || N == 0 || num_groups == 0) return chk;
@@ -66,6 +77,15 @@ extern "C" hif4_status hif4_grouped_gemm(const void* A_units, const void* B_unit
                           static_cast<size_t>(total_rows), st) != cudaSuccess)
       return HIF4_ERR_CUDA;
     return HIF4_OK;
+  }
+  const bool tc_ok = g_gemm_path != 1 &&
+                     gemm_tc_supported(A_units, B_units, total_rows, static_cast<int64_t>(num_groups) * N, N, K);
+  if (tc_ok) {
+    const size_t need = grouped_tc_workspace_bytes(num_groups, total_rows);
+    if (!workspace || workspace_bytes < need) return HIF4_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return HIF4_ERR_ALIGN;
+    return launch_grouped_gemm_tc(A_units, B_units, C, group_offsets_dev, num_groups, total_rows, N, K, ldc,
+                                  workspace, st);
   }
   return launch_grouped_gemm_simt(A_units, B_units, C, group_offsets_dev, num_groups, total_rows, N, K, ldc,
                                   st);

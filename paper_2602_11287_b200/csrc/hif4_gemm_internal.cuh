@@ -11,4 +11,13 @@ hif4_status launch_grouped_gemm_simt(const void* A, const void* B, float* C, con
                                      int num_groups, int64_t total_rows, int64_t N, int64_t K, int64_t ldc,
                                      cudaStream_t st);
 
+// Tensor-core path (tcgen05 + TMA): needs K % 256 == 0 and 16-byte aligned operands.
+bool gemm_tc_supported(const void* A, const void* B, int64_t a_rows, int64_t b_rows, int64_t N, int64_t K);
+hif4_status launch_gemm_tc(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,
+                           cudaStream_t st);
+size_t grouped_tc_workspace_bytes(int num_groups, int64_t total_rows);
+hif4_status launch_grouped_gemm_tc(const void* A, const void* B, float* C, const int64_t* offsets, int num_groups,
+                                   int64_t total_rows, int64_t N, int64_t K, int64_t ldc, void* workspace,
+                                   cudaStream_t st);
+
 }  // namespace hif4

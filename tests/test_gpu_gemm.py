@@ -118,7 +118,8 @@ def _grouped_case(hif4, counts, N, K, seed):
     a = hif4.hif4_quantize(torch.randn(max(total, 1), K, generator=g, device="cuda").to(torch.bfloat16))[:total]
     b = hif4.hif4_quantize((torch.randn(G * N, K, generator=g, device="cuda") * 0.02).to(torch.bfloat16)).view(G, N, K // 64, 36)
     out = torch.full((total, N), 3.0, dtype=torch.float32, device="cuda")
-    hif4.hif4_grouped_gemm(a, b, off.cuda(), out=out)
+    if total:
+        hif4.hif4_grouped_gemm(a, b, off.cuda(), out=out)
     ref, refabs = oracle.grouped_gemm_f64(a.cpu().numpy(), b.cpu().numpy(), off.numpy(), nthreads=8)
     err = np.abs(out.cpu().numpy().astype(np.float64) - ref)
     assert np.all(err <= TOL * refabs + 1e-300)
@@ -141,3 +142,62 @@ def test_grouped_gemm_moe_routing_sampled(hif4):
     ref, refabs = oracle.grouped_gemm_f64(a.cpu().numpy(), b.cpu().numpy(), off.cpu().numpy(), nthreads=8)
     err = np.abs(out.cpu().numpy().astype(np.float64) - ref)
     assert np.all(err <= TOL * refabs + 1e-300)
+
+
+# ------------------------------------------------------------------ tensor-core (tcgen05) kernel
+@pytest.fixture()
+def tc_path(hif4):
+    hif4.hif4_set_gemm_path(2)
+    yield hif4
+    hif4.hif4_set_gemm_path(0)
+    assert hif4.hif4_last_device_status() == 0, "a bounded wait inside the kernel ran out"
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 256, 256), (128, 256, 512), (1, 64, 256), (130, 257, 768), (300, 700, 1024),
+                                   (64, 2000, 256), (1000, 130, 2048)])
+def test_tensor_core_kernel_full_compare(tc_path, M, N, K):
+    hif4 = tc_path
+    g = torch.Generator(device="cuda"); g.manual_seed(M * 7 + N)
+    a = torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16)
+    b = (torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16)
+    before = hif4.launch_count()
+    C = check_full(hif4, hif4.hif4_quantize(a), hif4.hif4_quantize(b), f"tc {M}x{N}x{K}")
+    assert hif4.launch_count() - before == 3
+    C2 = hif4.hif4_gemm(hif4.hif4_quantize(a), hif4.hif4_quantize(b))
+    assert torch.equal(C, C2), "two runs of the tensor-core kernel differ"
+
+
+def test_tensor_core_kernel_random_units_nan_and_guard_bands(tc_path):
+    hif4 = tc_path
+    rng = np.random.default_rng(51)
+    M, N, upr = 150, 280, 8
+    A = rng.integers(0, 256, (M, upr, 36), dtype=np.uint8)
+    B = rng.integers(0, 256, (N, upr, 36), dtype=np.uint8)
+    A[..., 0] = rng.integers(0x00, 0xFF, (M, upr)); B[..., 0] = rng.integers(0x40, 0xC0, (N, upr))
+    A[77, 3, 0] = 0xFF
+    B[279, 7, 0] = 0xFF
+    out = torch.full((M + 2, 288), -5.0, dtype=torch.float32, device="cuda")
+    a, b = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+    C = hif4.hif4_gemm(a, b, out=out[1:M + 1, :N])
+    ref, refabs = oracle.gemm_f64(A, B, nthreads=8)
+    got = C.cpu().numpy().astype(np.float64)
+    nan = np.isnan(ref)
+    assert np.array_equal(np.isnan(got), nan)
+    err = np.abs(got - ref)[~nan]
+    assert np.all(err <= TOL * refabs[~nan] + 1e-300)
+    assert (out[0] == -5.0).all() and (out[M + 1] == -5.0).all() and (out[:, N:] == -5.0).all()
+
+
+def test_tensor_core_grouped(tc_path):
+    hif4 = tc_path
+    _grouped_case(hif4, [3, 0, 70, 1, 0, 129, 64, 0, 300], N=300, K=256, seed=61)
+    _grouped_case(hif4, [0, 0, 5], N=64, K=512, seed=62)
+    _grouped_case(hif4, [513], N=256, K=256, seed=63)
+
+
+def test_tensor_core_prefill_shape_sampled(tc_path):
+    hif4 = tc_path
+    K, N, M = 4096, 4096, 4096
+    w = hif4.hif4_quantize(wl.gaussian(N, K, 0.02, seed=71, device="cuda"))
+    x = hif4.hif4_quantize(wl.llama_activations(M, K, device="cuda"))
+    check_sampled(hif4, x, w, "tc llama qo M=4096", n=400)
