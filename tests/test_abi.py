@@ -1,0 +1,83 @@
+"""The C-ABI boundary without a GPU: libhif4.so loads, exports every function that include/hif4.h
+declares (and the Python binding lists the same names), and its host-only entry points answer as the
+header says.  No kernel is launched here."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "hif4.h")
+
+
+def declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    text = re.sub(r"typedef\s+enum\s*\{.*?\}\s*\w+\s*;", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(hif4_\w+)\s*\(", text)))
+
+
+@pytest.fixture(scope="module")
+def cdll():
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("_hif4_build", os.path.join(ROOT, "paper_2602_11287_b200", "build.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    return ctypes.CDLL(mod.build())
+
+
+def test_header_declares_the_calls_of_the_hot_path():
+    names = declared_functions()
+    for must in ("hif4_quantize", "hif4_dequantize", "hif4_gemm", "hif4_grouped_gemm", "hif4_packed_bytes",
+                 "hif4_gemm_workspace", "hif4_grouped_gemm_workspace", "hif4_last_device_status", "hif4_status_string"):
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol(cdll):
+    for name in declared_functions():
+        assert hasattr(cdll, name), f"libhif4.so does not export {name}"
+
+
+def test_binding_lists_the_same_names():
+    import paper_2602_11287_b200 as hif4
+    assert sorted(hif4.EXPORTED_SYMBOLS) == declared_functions()
+
+
+def test_host_only_entry_points(cdll):
+    i64, sz = ctypes.c_int64, ctypes.c_size_t
+    cdll.hif4_packed_bytes.restype = sz
+    cdll.hif4_packed_bytes.argtypes = [i64, i64]
+    assert cdll.hif4_packed_bytes(3, 128) == 3 * 2 * 36            # 288 bits per 64 values (Section II-A)
+    assert cdll.hif4_packed_bytes(1, 64) * 8 == 288
+    assert cdll.hif4_packed_bytes(3, 100) == 0 and cdll.hif4_packed_bytes(-1, 64) == 0
+    cdll.hif4_status_string.restype = ctypes.c_char_p
+    seen = {cdll.hif4_status_string(c) for c in range(9)}
+    assert len(seen) == 9 and all(s for s in seen)
+    n = sz(123)
+    cdll.hif4_gemm_workspace.argtypes = [i64, i64, i64, ctypes.POINTER(sz)]
+    assert cdll.hif4_gemm_workspace(16, 16, 128, ctypes.byref(n)) == 0
+    assert cdll.hif4_gemm_workspace(16, 16, 100, ctypes.byref(n)) == 2          # K % 64
+    assert cdll.hif4_gemm_workspace(16, 16, 128, None) == 1
+    cdll.hif4_grouped_gemm_workspace.argtypes = [ctypes.c_int, i64, i64, i64, ctypes.POINTER(sz)]
+    assert cdll.hif4_grouped_gemm_workspace(4, 1000, 256, 512, ctypes.byref(n)) == 0
+    assert n.value >= (1000 // 128 + 4) * 16 and n.value % 256 == 0
+    assert cdll.hif4_grouped_gemm_workspace(-1, 10, 64, 64, ctypes.byref(n)) == 2
+
+
+def test_argument_errors_are_found_before_any_launch(cdll):
+    """Shape / dtype / null checks come before the first CUDA call, so they answer without a GPU."""
+    i64, vp, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
+    cdll.hif4_quantize.argtypes = [vp, ci, i64, i64, i64, vp, ci, vp]
+    cdll.hif4_launch_count.restype = ctypes.c_uint64
+    before = cdll.hif4_launch_count()
+    assert cdll.hif4_quantize(None, 0, 4, 100, 100, None, 0, None) == 2     # cols % 64
+    assert cdll.hif4_quantize(None, 5, 4, 128, 128, None, 0, None) == 4     # dtype
+    assert cdll.hif4_quantize(None, 0, 4, 128, 128, None, 9, None) == 4     # rounding mode
+    assert cdll.hif4_quantize(None, 0, 4, 128, 64, None, 0, None) == 2      # ld < cols
+    assert cdll.hif4_quantize(None, 0, 4, 128, 128, None, 0, None) == 1     # null
+    assert cdll.hif4_quantize(None, 0, 0, 128, 128, None, 0, None) == 0     # empty: no-op
+    cdll.hif4_gemm.argtypes = [vp, vp, vp, i64, i64, i64, i64, vp, ctypes.c_size_t, vp]
+    assert cdll.hif4_gemm(None, None, None, 4, 4, 100, 4, None, 0, None) == 2
+    assert cdll.hif4_gemm(None, None, None, 0, 4, 64, 4, None, 0, None) == 0
+    assert cdll.hif4_launch_count() == before
