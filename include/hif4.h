@@ -123,6 +123,37 @@ hif4_status hif4_grouped_gemm(const void* A_units, const void* B_units, float* C
                               int64_t N, int64_t K, int64_t ldc, void* workspace,
                               size_t workspace_bytes, void* stream);
 
+/* hif4_grouped_gemm_noalloc -- hif4_grouped_gemm without a workspace argument.  (The paper has no
+ * counterpart: this is a packaging variant of the call above, not another operation.)
+ *
+ * For callers that cannot allocate device memory: code running under a fixed memory plan that was
+ * sized at start-up, a plug-in that receives tensors but no allocator, or a section where the
+ * device-wide synchronisation of a cudaMalloc is not acceptable.  The tile table that the
+ * tensor-core kernel needs lives in a __device__ array of HIF4_NOALLOC_SCRATCH_BYTES bytes inside
+ * the library; every GPU that loads the library holds it until the process exits.  The call itself
+ * performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ *   Arguments and result are those of hif4_grouped_gemm (same kernels, same bits in C).
+ *   Limit     ceil(total_rows / 128) + num_groups table entries of 16 bytes, rounded up to 256,
+ *             must fit in HIF4_NOALLOC_SCRATCH_BYTES (65536: e.g. 256 groups and 491520 rows);
+ *             beyond that the call returns HIF4_ERR_WORKSPACE and launches nothing.
+ *   Sharing   all calls on one GPU use the same array.  Calls ordered on one stream are safe (each
+ *             call rewrites every entry it reads; nothing has to be zero beforehand).  Calls that
+ *             may overlap on the GPU -- different streams or host threads without ordering -- race
+ *             on the table and produce wrong results.
+ *   Set-up    the first call on each GPU looks up the array's device address
+ *             (cudaGetSymbolAddress, with that GPU current) and keeps it; make that first call
+ *             outside any stream capture.
+ * hif4_set_gemm_path does not apply to this call.  */
+#define HIF4_NOALLOC_SCRATCH_BYTES 65536
+hif4_status hif4_grouped_gemm_noalloc(const void* A_units, const void* B_units, float* C,
+                                      const int64_t* group_offsets_dev, int num_groups,
+                                      int64_t total_rows, int64_t N, int64_t K, int64_t ldc,
+                                      void* stream);
+
+/* Size in bytes of the built-in scratch array (HIF4_NOALLOC_SCRATCH_BYTES).  Host-only.  */
+size_t hif4_grouped_gemm_noalloc_capacity(void);
+
 /* Synchronises `stream` and returns HIF4_ERR_DEVICE_TIMEOUT if any kernel of this library gave up
  * a bounded wait since the last call (the flag is cleared), HIF4_ERR_CUDA if the stream reports
  * an error, else HIF4_OK.  For tests and debugging.  */

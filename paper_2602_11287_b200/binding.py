@@ -23,7 +23,7 @@ HIF4_OK = 0
 EXPORTED_SYMBOLS = [
     "hif4_packed_bytes", "hif4_quantize", "hif4_dequantize", "hif4_gemm_workspace", "hif4_gemm",
     "hif4_grouped_gemm_workspace", "hif4_grouped_gemm", "hif4_last_device_status", "hif4_status_string",
-    "hif4_launch_count", "hif4_set_gemm_path",
+    "hif4_launch_count", "hif4_set_gemm_path", "hif4_grouped_gemm_noalloc", "hif4_grouped_gemm_noalloc_capacity",
 ]
 
 
@@ -54,6 +54,10 @@ def _load() -> ctypes.CDLL:
     L.hif4_grouped_gemm_workspace.argtypes = [ci, i64, i64, i64, ctypes.POINTER(sz)]
     L.hif4_grouped_gemm.restype = ci
     L.hif4_grouped_gemm.argtypes = [vp, vp, vp, vp, ci, i64, i64, i64, i64, vp, sz, vp]
+    L.hif4_grouped_gemm_noalloc.restype = ci
+    L.hif4_grouped_gemm_noalloc.argtypes = [vp, vp, vp, vp, ci, i64, i64, i64, i64, vp]
+    L.hif4_grouped_gemm_noalloc_capacity.restype = sz
+    L.hif4_grouped_gemm_noalloc_capacity.argtypes = []
     L.hif4_last_device_status.restype = ci
     L.hif4_last_device_status.argtypes = [vp]
     L.hif4_status_string.restype = ctypes.c_char_p
@@ -195,6 +199,32 @@ def hif4_grouped_gemm(a_units: torch.Tensor, b_units: torch.Tensor, group_offset
            lib.hif4_grouped_gemm(a_units.data_ptr(), b_units.data_ptr(), out.data_ptr(), group_offsets.data_ptr(),
                                  G, total, N, K, ldc, workspace.data_ptr() if workspace is not None else None,
                                  workspace.numel() if workspace is not None else 0, _stream(stream)))
+    return out
+
+
+def hif4_grouped_gemm_noalloc_capacity() -> int:
+    """Bytes of the scratch array built into the library for `hif4_grouped_gemm_noalloc`."""
+    return int(lib.hif4_grouped_gemm_noalloc_capacity())
+
+
+def hif4_grouped_gemm_noalloc(a_units: torch.Tensor, b_units: torch.Tensor, group_offsets: torch.Tensor,
+                              out: torch.Tensor, stream=None) -> torch.Tensor:
+    """`hif4_grouped_gemm` for callers that may not allocate on the device: the output must be passed
+    in, and the kernel's tile table sits in a fixed array inside the library instead of a workspace.
+    Problems whose table does not fit are refused (Hif4Error, status 5).  All calls on a GPU share
+    that array, so calls that could overlap on the GPU must be ordered by the caller."""
+    _need_cuda(a_units, b_units, group_offsets, out)
+    assert a_units.dtype == torch.uint8 and b_units.dtype == torch.uint8 and group_offsets.dtype == torch.int64
+    assert a_units.dim() == 3 and b_units.dim() == 4 and a_units.shape[1] == b_units.shape[2]
+    assert a_units.is_contiguous() and b_units.is_contiguous() and group_offsets.is_contiguous()
+    total, upr, _ = a_units.shape
+    G, N = b_units.shape[0], b_units.shape[1]
+    assert group_offsets.numel() == G + 1
+    assert out.dtype == torch.float32 and out.stride(1) == 1 and out.shape == (total, N)
+    ldc = out.stride(0) if total > 1 else max(N, out.stride(0))
+    _check("hif4_grouped_gemm_noalloc",
+           lib.hif4_grouped_gemm_noalloc(a_units.data_ptr(), b_units.data_ptr(), out.data_ptr(),
+                                         group_offsets.data_ptr(), G, total, N, upr * UNIT_ELEMS, ldc, _stream(stream)))
     return out
 
 
