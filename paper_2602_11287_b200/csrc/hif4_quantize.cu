@@ -2,10 +2,9 @@
 // streaming CUDA kernels for sm_100a.  Both are bound by HBM traffic: 2 B (or 4 B) read and
 // 0.5625 B written per element for the quantizer, the reverse for the dequantizer.
 //
-// BF16 quantizer, thread mapping: 8 consecutive lanes own one 64-element unit; lane j loads the
-// 16 bytes of level-2 group j (elements 8j..8j+7) with one 128-bit load, so a warp reads 512
-// contiguous bytes (4 units) per load instruction and each lane issues kUnroll loads before it
-// computes.  Algorithm 1 is written in BF16 arithmetic; packed bf16x2 instructions with
+// BF16 quantizer, thread mapping: 4 consecutive lanes own one 64-element unit; lane q loads the
+// 16 bytes of level-2 groups q and q + 4 (elements 8q..8q+7 and 32+8q..) with two 128-bit loads, so
+// a warp covers 8 units per pass and each lane issues 2 * kUnroll loads before it computes.  Algorithm 1 is written in BF16 arithmetic; packed bf16x2 instructions with
 // round-to-nearest-even are exactly that arithmetic for two elements at a time:
 //   - peak magnitudes are integer maxima of the |x| bit patterns (NaN patterns sort above Inf);
 //   - SF = Vmax * (1/7)_BF16 is one mul.rn.bf16x2; rounding SF to the 3-bit-significand E6M2 byte is
@@ -84,94 +83,115 @@ __device__ __forceinline__ int64_t unit_offset(int64_t u, int64_t upr, int64_t l
 }
 
 // ----------------------------------------------------------------------------- BF16 quantizer
+// Stage 3 of Algorithm 1 for one level-2 group (8 elements, magnitudes a0..a3 as bf16x2 pairs, source
+// words x0..x3 for the signs): micro-exponents from the peaks of the products, S1P2 codes packed into
+// one 32-bit word.  `e8`, `e16a`, `e16b` come back as 0/1.
+template <bool kRHA>
+__device__ __forceinline__ uint32_t encode_group_bf16(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3,
+                                                      uint32_t rec2, uint32_t& e8, uint32_t& e16a,
+                                                      uint32_t& e16b) {
+  const uint32_t t0 = mul_bf16x2(x0 & 0x7FFF7FFFu, rec2), t1 = mul_bf16x2(x1 & 0x7FFF7FFFu, rec2),
+                 t2 = mul_bf16x2(x2 & 0x7FFF7FFFu, rec2), t3 = mul_bf16x2(x3 & 0x7FFF7FFFu, rec2);
+  const uint32_t p16a = hmax_halves(umax2(t0, t1));     // elements 0..3 of the group
+  const uint32_t p16b = hmax_halves(umax2(t2, t3));     // elements 4..7
+  e8 = max(p16a, p16b) >= 0x4080u;                      // >= 4.0
+  const uint32_t thr = 0x4000u + (e8 << 7);             // 2.0 * 2^e8
+  e16a = p16a >= thr;
+  e16b = p16b >= thr;
+  uint32_t c0, c1, c2, c3;
+  if (!kRHA) {
+    // quarter counts 4 * t * 2^-(e8+e16) rounded to nearest-even in the low mantissa bits of 128 + q
+    const uint32_t mula = 0x40804080u - (e8 + e16a) * 0x00800080u;
+    const uint32_t mulb = 0x40804080u - (e8 + e16b) * 0x00800080u;
+    c0 = __vminu2(fma_bf16x2(t0, mula, 0x43004300u), 0x43074307u);
+    c1 = __vminu2(fma_bf16x2(t1, mula, 0x43004300u), 0x43074307u);
+    c2 = __vminu2(fma_bf16x2(t2, mulb, 0x43004300u), 0x43074307u);
+    c3 = __vminu2(fma_bf16x2(t3, mulb, 0x43004300u), 0x43074307u);
+  } else {
+    // round-half-away: widen to FP32 (exact), add one half, truncate
+    const float fa = __uint_as_float((129u - (e8 + e16a)) << 23);
+    const float fb = __uint_as_float((129u - (e8 + e16b)) << 23);
+    auto rha = [](uint32_t t, float f) {
+      const float lo = fminf(__uint_as_float(t << 16) * f, 8.0f);
+      const float hi = fminf(__uint_as_float(t & 0xFFFF0000u) * f, 8.0f);
+      const uint32_t ql = min(static_cast<uint32_t>(lo + 0.5f), 7u);
+      const uint32_t qh = min(static_cast<uint32_t>(hi + 0.5f), 7u);
+      return 0x43004300u | ql | (qh << 16);
+    };
+    c0 = rha(t0, fa); c1 = rha(t1, fa); c2 = rha(t2, fb); c3 = rha(t3, fb);
+  }
+  // Pack: low bytes of the four bf16x2 results hold the magnitudes; signs come from the top bit of
+  // each source element.  Pairs are gathered in swapped order so that one multiply by 0x1001
+  // drops (q_even | q_odd << 4) into bytes 1 and 3.
+  uint32_t g0 = prmt(c0, c1, 0x4602u), g1 = prmt(c2, c3, 0x4602u);
+  g0 |= prmt(x0, x1, 0xDF9Bu) & 0x08080808u;
+  g1 |= prmt(x2, x3, 0xDF9Bu) & 0x08080808u;
+  return prmt(g0 * 0x1001u, g1 * 0x1001u, 0x7531u);
+}
+
+// Four consecutive lanes own one unit: lane q loads the 16-byte chunks q and q + 4 of its 128 bytes,
+// i.e. the level-2 groups q and q + 4, so that each load instruction of a warp reads eight 64-byte
+// runs and the per-unit scalar work (scale, reciprocal) is shared by 16 elements.  A warp handles 8
+// units per pass and issues all 2 * kUnroll loads before it computes.
 template <bool kRHA, bool kContig>
 __global__ void __launch_bounds__(kThreads)
 quantize_bf16_kernel(const uint16_t* __restrict__ src, int64_t n_units, int64_t upr, int64_t ld_src,
                      uint32_t* __restrict__ dst) {
   const int lane = threadIdx.x & 31;
-  const int j = lane & 7;                    // level-2 group owned by this lane
+  const int q = lane & 3;
   const int64_t warp = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) >> 5;
-  const int64_t first = warp * (4 * kUnroll) + (lane >> 3);
+  const int64_t first = warp * (8 * kUnroll) + (lane >> 2);
+  // metadata bit weights of this lane's two groups: E1_8 bits 8+q, 12+q; E1_16 bits 16+2q(+1), 24+2q(+1)
+  const uint32_t w8 = 0x100u << q, w16 = 0x10000u << (2 * q);
 
-  uint4 v[kUnroll];
+  uint4 va[kUnroll], vb[kUnroll];
 #pragma unroll
   for (int i = 0; i < kUnroll; ++i) {
-    const int64_t u = first + 4 * i;
-    v[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (u < n_units)
-      v[i] = ld_stream(reinterpret_cast<const uint4*>(src + unit_offset<kContig>(u, upr, ld_src) + 8 * j));
+    const int64_t u = first + 8 * i;
+    va[i] = make_uint4(0u, 0u, 0u, 0u);
+    vb[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (u < n_units) {
+      const uint4* p = reinterpret_cast<const uint4*>(src + unit_offset<kContig>(u, upr, ld_src)) + q;
+      va[i] = ld_stream(p);
+      vb[i] = ld_stream(p + 4);
+    }
   }
 
 #pragma unroll
   for (int i = 0; i < kUnroll; ++i) {
-    const int64_t u = first + 4 * i;
-    const uint32_t x0 = v[i].x, x1 = v[i].y, x2 = v[i].z, x3 = v[i].w;
-    const uint32_t a0 = x0 & 0x7FFF7FFFu, a1 = x1 & 0x7FFF7FFFu, a2 = x2 & 0x7FFF7FFFu,
-                   a3 = x3 & 0x7FFF7FFFu;
-    // Stage 1: peak magnitude of the unit (the group peaks are taken on the products below).
-    uint32_t vm = hmax_halves(umax2(umax2(a0, a1), umax2(a2, a3)));
+    const int64_t u = first + 8 * i;
+    // Stage 1: peak magnitude of the unit as an integer maximum of the |x| bit patterns (the group
+    // peaks are taken on the products in encode_group_bf16).
+    constexpr uint32_t kAbs = 0x7FFF7FFFu;
+    uint32_t vm = umax2(umax2(umax2(va[i].x & kAbs, va[i].y & kAbs), umax2(va[i].z & kAbs, va[i].w & kAbs)),
+                        umax2(umax2(vb[i].x & kAbs, vb[i].y & kAbs), umax2(vb[i].z & kAbs, vb[i].w & kAbs)));
+    vm = hmax_halves(vm);
     vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 1));
     vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 2));
-    vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 4));
     const bool unit_nan = vm > 0x7F80u;
 
     // Stage 2: level-1 scale, its reciprocal.
     const uint32_t sf = mul_bf16x2(vm, 0x3E12u) & 0xFFFFu;             // Vmax * (1/7)_BF16
     const uint32_t byte = e6m2_from_bits<7, kRHA>(sf);
-    const uint32_t lut = (0x122B4D80u >> ((byte & 3u) * 8u)) & 0xFFu;   // 1/1.M in BF16: 3F80 3F4D 3F2B 3F12
-    const uint32_t rec = (0x3F00u | lut) + (48u << 7) - ((byte >> 2) << 7);
-    const uint32_t rec2 = rec * 0x10001u;
+    // 1/1.M in BF16 is 3F80 3F4D 3F2B 3F12: low byte by table, then the exponent subtraction
+    const uint32_t lut = prmt(0x122B4D80u, 0u, (byte & 3u) | 0x4440u);
+    const uint32_t rec2 = (lut + 0x5700u - ((byte & 0xFCu) << 5)) * 0x10001u;
 
-    const uint32_t t0 = mul_bf16x2(a0, rec2), t1 = mul_bf16x2(a1, rec2), t2 = mul_bf16x2(a2, rec2),
-                   t3 = mul_bf16x2(a3, rec2);
-    // Level-2 and level-3 micro-exponents from the peaks of the products.
-    const uint32_t p16a = hmax_halves(umax2(t0, t1));     // elements 0..3 of this lane
-    const uint32_t p16b = hmax_halves(umax2(t2, t3));     // elements 4..7
-    const uint32_t e8 = max(p16a, p16b) >= 0x4080u;       // >= 4.0
-    const uint32_t thr = 0x4000u + (e8 << 7);             // 2.0 * 2^e8
-    const uint32_t e16a = p16a >= thr, e16b = p16b >= thr;
+    uint32_t e8a, e16a0, e16a1, e8b, e16b0, e16b1;
+    uint32_t codes_a = encode_group_bf16<kRHA>(va[i].x, va[i].y, va[i].z, va[i].w, rec2, e8a, e16a0, e16a1);
+    uint32_t codes_b = encode_group_bf16<kRHA>(vb[i].x, vb[i].y, vb[i].z, vb[i].w, rec2, e8b, e16b0, e16b1);
 
-    // Stage 3: quarter counts 4 * t * 2^-(e8+e16), rounded, clamped to 7.
-    uint32_t c0, c1, c2, c3;
-    if (!kRHA) {
-      const uint32_t mula = (0x4080u - ((e8 + e16a) << 7)) * 0x10001u;
-      const uint32_t mulb = (0x4080u - ((e8 + e16b) << 7)) * 0x10001u;
-      c0 = __vminu2(fma_bf16x2(t0, mula, 0x43004300u), 0x43074307u);
-      c1 = __vminu2(fma_bf16x2(t1, mula, 0x43004300u), 0x43074307u);
-      c2 = __vminu2(fma_bf16x2(t2, mulb, 0x43004300u), 0x43074307u);
-      c3 = __vminu2(fma_bf16x2(t3, mulb, 0x43004300u), 0x43074307u);
-    } else {
-      // round-half-away: widen to FP32 (exact), add one half, truncate
-      const float fa = __uint_as_float((129u - (e8 + e16a)) << 23);
-      const float fb = __uint_as_float((129u - (e8 + e16b)) << 23);
-      auto rha = [](uint32_t t, float f) {
-        const float lo = fminf(__uint_as_float(t << 16) * f, 8.0f);
-        const float hi = fminf(__uint_as_float(t & 0xFFFF0000u) * f, 8.0f);
-        const uint32_t ql = min(static_cast<uint32_t>(lo + 0.5f), 7u);
-        const uint32_t qh = min(static_cast<uint32_t>(hi + 0.5f), 7u);
-        return 0x43004300u | ql | (qh << 16);
-      };
-      c0 = rha(t0, fa); c1 = rha(t1, fa); c2 = rha(t2, fb); c3 = rha(t3, fb);
-    }
-    // Pack: low bytes of the four bf16x2 results hold the magnitudes; signs come from the top bit of
-    // each source element.  Pairs are gathered in swapped order so that one multiply by 0x1001
-    // drops (q_even | q_odd << 4) into bytes 1 and 3.
-    uint32_t g0 = prmt(c0, c1, 0x4602u), g1 = prmt(c2, c3, 0x4602u);
-    g0 |= prmt(x0, x1, 0xDF9Bu) & 0x08080808u;
-    g1 |= prmt(x2, x3, 0xDF9Bu) & 0x08080808u;
-    uint32_t codes = prmt(g0 * 0x1001u, g1 * 0x1001u, 0x7531u);
-
-    uint32_t meta = (e8 << (8 + j)) | (e16a << (16 + 2 * j)) | (e16b << (17 + 2 * j));
+    uint32_t meta = (e8a + (e8b << 4)) * w8 + (e16a0 + 2u * e16a1 + ((e16b0 + 2u * e16b1) << 8)) * w16;
     meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 1);
     meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 2);
-    meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 4);
     meta |= byte;
-    if (unit_nan) { meta = 0xFFu; codes = 0u; }          // NaN unit: E6M2 = NaN, everything else zero
+    if (unit_nan) { meta = 0xFFu; codes_a = 0u; codes_b = 0u; }   // NaN unit: E6M2 = NaN, all else zero
 
     if (u < n_units) {
       uint32_t* out = dst + u * kUnitWords;
-      st_stream(out + 1 + j, codes);
-      if (j == 0) st_stream(out, meta);
+      st_stream(out + 1 + q, codes_a);
+      st_stream(out + 5 + q, codes_b);
+      if (q == 0) st_stream(out, meta);
     }
   }
 }
@@ -334,7 +354,7 @@ extern "C" hif4_status hif4_quantize(const void* src, hif4_dtype dt, int64_t row
   const int64_t upr = cols / kUnitElems;
   const int64_t n_units = rows * upr;
   const bool contig = ld_src == cols;
-  const int units_per_block = (kThreads / 32) * kUnroll * (dt == HIF4_BF16 ? 4 : 2);
+  const int units_per_block = (kThreads / 32) * kUnroll * (dt == HIF4_BF16 ? 8 : 2);
   const int64_t blocks = ceil_div64(n_units, units_per_block);
   if (blocks > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
