@@ -163,8 +163,9 @@ hif4_status hif4_last_device_status(void* stream);
 const char* hif4_status_string(hif4_status s);
 
 /* Diagnostic: 0 = choose the GEMM kernel by shape (default), 1 = CUDA-core kernel only, 2 = the
- * tensor-core (tcgen05) kernel whenever it is legal (K % 256 == 0, 16-byte aligned operands), even
- * for small M.  Process-wide, not thread-safe; meant for tests and benchmarks.  */
+ * single-CTA tensor-core (tcgen05) kernel whenever it is legal (K % 256 == 0, 16-byte aligned
+ * operands), even for small M, 3 = the CTA-pair tensor-core kernel (256 x 256 tiles) whenever it is
+ * legal.  Process-wide, not thread-safe; meant for tests and benchmarks.  */
 hif4_status hif4_set_gemm_path(int path);
 
 /* Number of kernels this library has launched in this process (monotonic, host-side counter).  */

@@ -5,9 +5,11 @@
 using namespace hif4;
 
 namespace {
-// 0 = choose by shape, 1 = CUDA-core kernel only, 2 = tensor-core kernel whenever it is legal.
+// 0 = choose by shape, 1 = CUDA-core kernel only, 2 = single-CTA tensor-core kernel whenever it is
+// legal, 3 = CTA-pair tensor-core kernel whenever it is legal.
 int g_gemm_path = 0;
 constexpr int64_t kTensorCoreMinM = 64;
+constexpr int64_t kPairMinM = 129;      // below that a 256-row pair tile would be half empty
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -29,7 +31,7 @@ extern "C" hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size
 }
 
 extern "C" hif4_status hif4_set_gemm_path(int path) {
-  if (path < 0 || path > 2) return HIF4_ERR_DTYPE;
+  if (path < 0 || path > 3) return HIF4_ERR_DTYPE;
   g_gemm_path = path;
   return HIF4_OK;
 }
@@ -49,7 +51,9 @@ extern "C" hif4_status hif4_gemm(const void* A_units, const void* B_units, float
     return HIF4_OK;
   }
   const bool tc_ok = g_gemm_path != 1 && gemm_tc_supported(A_units, B_units, M, N, N, K);
-  if (tc_ok && (g_gemm_path == 2 || M >= kTensorCoreMinM)) return launch_gemm_tc(A_units, B_units, C, M, N, K, ldc, st);
+  if (tc_ok && g_gemm_path != 2 && (g_gemm_path == 3 || M >= kPairMinM) && gemm_tc2_supported(A_units, B_units, M, N, K))
+    return launch_gemm_tc2(A_units, B_units, C, M, N, K, ldc, st);
+  if (tc_ok && (g_gemm_path >= 2 || M >= kTensorCoreMinM)) return launch_gemm_tc(A_units, B_units, C, M, N, K, ldc, st);
   return launch_gemm_simt(A_units, B_units, C, M, N, K, ldc, st);
 }
 

@@ -15,6 +15,10 @@ hif4_status launch_grouped_gemm_simt(const void* A, const void* B, float* C, con
 bool gemm_tc_supported(const void* A, const void* B, int64_t a_rows, int64_t b_rows, int64_t N, int64_t K);
 hif4_status launch_gemm_tc(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,
                            cudaStream_t st);
+// Tensor-core path on CTA pairs (256 x 256 tiles, tcgen05 cta_group::2): same requirements.
+bool gemm_tc2_supported(const void* A, const void* B, int64_t M, int64_t N, int64_t K);
+hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,
+                            cudaStream_t st);
 size_t grouped_tc_workspace_bytes(int num_groups, int64_t total_rows);
 hif4_status launch_grouped_gemm_tc(const void* A, const void* B, float* C, const int64_t* offsets, int num_groups,
                                    int64_t total_rows, int64_t N, int64_t K, int64_t ldc, void* workspace,

@@ -1,0 +1,357 @@
+// Tensor-core HiF4 x HiF4 -> FP32 GEMM for sm_100a on CTA pairs: C = A * B^T (Eq. 3 summed over unit
+// pairs), 256 x 256 output tile per pair of SMs (tcgen05.mma cta_group::2).
+//
+// Same arithmetic as the single-CTA kernel (every HiF4 value, level-1 scale included, is exactly a
+// BF16; products are exact in the FP32 accumulator), different work split.  The cost that bounds
+// this GEMM is the decode of packed units into BF16 operand tiles on the CUDA cores; a 128 x 256 tile
+// on one SM decodes 128 + 256 rows per 64-wide K block, a 256 x 256 tile on two SMs only 128 + 128 rows
+// per SM for the same tensor work per SM.  Cluster of two CTAs, rank r:
+//   warp 0       TMA producer: raw units of A rows [m0 + 128 r, +128) and B rows [n0 + 128 r, +128),
+//                4 units (K = 256, 144 bytes) per row per stage, two stages; each CTA fetches its own rows
+//   warps 6-21   decode: 512 threads = 256 tile rows x 2; thread (row, h) loads 80 bytes of the row's
+//                raw chunk and decodes units 2h and 2h+1 (Eq. 2) into K-major SWIZZLE_128B operand
+//                rows of decoded stages 2h and 2h+1 (a K = 64 block each, four stages)
+//   warp 1       rank 0 only: issues tcgen05.mma.cta_group::2 (256 x 256 x 16, four per K block), which
+//                reads A and B halves from both CTAs' shared memory and accumulates into both CTAs'
+//                tensor memory; commits are multicast to the barriers of both CTAs
+//   warps 2-5    epilogue: tcgen05.ld of this CTA's 128 accumulator rows, FP32 stores to C
+// Cross-CTA signalling: "decoded stage full" and "accumulator drained" are mbarriers of rank 0 on which
+// the threads of both CTAs arrive (remote arrives with release at cluster scope); "stage free" and
+// "accumulator complete" arrive in both CTAs through the multicast commit.
+//
+// Every wait on an mbarrier is bounded: when the budget runs out the CTA raises an error word, every
+// role leaves its loop, both CTAs meet at the final cluster barrier, tensor memory is released and
+// the kernel returns.
+#include "hif4_common.cuh"
+#include "hif4_gemm_internal.cuh"
+#include "hif4_tc_common.cuh"
+
+namespace hif4 {
+namespace {
+
+constexpr int kPairM = 256, kPairN = 256;             // output tile of a CTA pair
+constexpr int kRows = 128;                            // A rows and B rows per CTA
+constexpr int kRawHalfBytes = kRows * kRawRowBytes;   // 18432
+constexpr int kRawStageBytes = 2 * kRawHalfBytes;     // A rows then B rows
+constexpr int kDecHalfBytes = kRows * 128;            // 128 rows x 64 BF16
+constexpr int kDecStageBytes = 2 * kDecHalfBytes;
+constexpr int kRawStages = 2;
+constexpr int kDecStages = 4;                         // one per unit of a raw chunk
+constexpr int kTmemCols = 512;                        // two 256-column accumulators
+
+constexpr int kDecodeWarp0 = 6;
+constexpr int kDecodeThreads = 4 * kRows;             // 512: (A rows + B rows) x 2 unit pairs
+constexpr int kThreads = kDecodeWarp0 * 32 + kDecodeThreads;   // 704
+
+constexpr int kSmemBytes = 1024 /*alignment slack*/ + kDecStages * kDecStageBytes + kRawStages * kRawStageBytes + 256;
+
+// tcgen05.mma kind::f16 instruction descriptor: D = F32, A = B = BF16, both K-major, N/8, M/16.
+constexpr uint32_t kInstrDesc2 = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kPairN >> 3) << 17) |
+                                 (static_cast<uint32_t>(kPairM >> 4) << 24);
+
+struct Gemm2Params {
+  float* C;
+  int64_t ldc;
+  int64_t M;
+  int64_t N;
+  int num_kc;           // K / 256
+  int n_tiles;          // ceil(N / 256)
+  int total_tiles;
+  unsigned int* error_word;
+};
+
+// ------------------------------------------------------------------------------ cluster-scope PTX
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait on a barrier that threads of the peer CTA arrive on.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_try_cluster(bar, parity)) return true;
+  const uint64_t t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_cluster(bar, parity)) return true;
+    if ((it & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > kWaitBudgetNs) {
+        *abort_flag = 1u;
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc2_commit_both(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+      "h"(static_cast<uint16_t>(3))
+      : "memory");
+}
+__device__ __forceinline__ void tc2_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+struct PairTile { int m0; int n0; };
+__device__ __forceinline__ PairTile pair_tile(const Gemm2Params& p, int t) {
+  const int mt = t / p.n_tiles;
+  return PairTile{mt * kPairM, (t - mt * p.n_tiles) * kPairN};
+}
+
+// Decodes the two units held in raw words L[kOff .. kOff+8] and L[kOff+9 .. kOff+17] into decoded
+// stages 2h and 2h+1.  Returns false when a wait gave up.
+template <int kOff>
+__device__ __forceinline__ bool decode_two_units(const uint32_t (&L)[20], uint32_t stage0_row_addr, uint32_t r7,
+                                                 uint32_t dec_empty0, uint32_t dec_full0_leader, uint32_t parity_free,
+                                                 volatile uint32_t* abort_flag) {
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    if (!mbar_wait(dec_empty0 + 8 * u, parity_free, abort_flag)) return false;
+    decode_unit_to_row(L[kOff + 9 * u], &L[kOff + 9 * u + 1], stage0_row_addr + u * kDecStageBytes, r7);
+    fence_proxy_async_smem();                  // generic-proxy writes -> visible to the tensor core
+    mbar_arrive_cluster(dec_full0_leader + 8 * u);
+  }
+  return true;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                const Gemm2Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t dec_base = smem_base;                                        // 1024-byte aligned stages
+  const uint32_t raw_base = dec_base + kDecStages * kDecStageBytes;
+  const uint32_t bar_base = raw_base + kRawStages * kRawStageBytes;
+  // barriers (8 bytes each)
+  const uint32_t raw_full = bar_base, raw_empty = bar_base + 16, dec_full = bar_base + 32, dec_empty = bar_base + 64,
+                 tmem_full = bar_base + 96, tmem_empty = bar_base + 112;
+  uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(gen_base + (bar_base - smem_base) + 128);
+  volatile uint32_t* abort_flag = tmem_ptr_smem + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kRawStages; ++s) {
+      mbar_init(raw_full + 8 * s, 1);
+      mbar_init(raw_empty + 8 * s, kDecodeThreads);
+    }
+    for (int s = 0; s < kDecStages; ++s) {
+      mbar_init(dec_full + 8 * s, kDecodeThreads);    // 256 threads of each CTA per stage (used on rank 0)
+      mbar_init(dec_empty + 8 * s, 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(tmem_full + 8 * s, 1);
+      mbar_init(tmem_empty + 8 * s, 256);             // 128 epilogue threads of each CTA (used on rank 0)
+    }
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bar_base + 128),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();            // the peer's barriers are initialised before anyone arrives on them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_ptr_smem;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      uint32_t n = 0;
+      bool ok = true;
+      for (int t = pair; t < p.total_tiles && ok; t += num_pairs) {
+        const PairTile tc = pair_tile(p, t);
+        for (int kc = 0; kc < p.num_kc; ++kc, ++n) {
+          const uint32_t s = n & 1u, ph = (n >> 1) & 1u;
+          if (!(ok = mbar_wait(raw_empty + 8 * s, ph ^ 1u, abort_flag))) break;
+          mbar_expect_tx(raw_full + 8 * s, kRawStageBytes);
+          const uint32_t dst = raw_base + s * kRawStageBytes;
+          tma_load_2d(dst, &tmA, kc * kRawRowBytes, tc.m0 + static_cast<int>(rank) * kRows, raw_full + 8 * s);
+          tma_load_2d(dst + kRawHalfBytes, &tmB, kc * kRawRowBytes, tc.n0 + static_cast<int>(rank) * kRows,
+                      raw_full + 8 * s);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer (rank 0 only)
+    if (rank == 0 && lane == 0) {
+      uint32_t n = 0, tcount = 0;
+      bool ok = true;
+      for (int t = pair; t < p.total_tiles && ok; t += num_pairs, ++tcount) {
+        const uint32_t acc = tcount & 1u, aph = (tcount >> 1) & 1u;
+        if (!(ok = mbar_wait_cluster(tmem_empty + 8 * acc, aph ^ 1u, abort_flag))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * kPairN;
+        for (int kc = 0; kc < p.num_kc && ok; ++kc, ++n) {
+#pragma unroll
+          for (int u = 0; u < kDecStages; ++u) {
+            if (!(ok = mbar_wait_cluster(dec_full + 8 * u, n & 1u, abort_flag))) break;
+            tc_fence_after();
+            const uint64_t adesc = make_desc(dec_base + u * kDecStageBytes);
+            const uint64_t bdesc = make_desc(dec_base + u * kDecStageBytes + kDecHalfBytes);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              tc2_mma(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, kInstrDesc2, (kc | u | kk) != 0 ? 1u : 0u);
+            tc2_commit_both(dec_empty + 8 * u);       // both CTAs may overwrite the stage once these MMAs have read it
+          }
+        }
+        if (!ok) break;
+        tc2_commit_both(tmem_full + 8 * acc);         // accumulator complete, in both CTAs
+      }
+    }
+  } else if (warp < kDecodeWarp0) {
+    // ---------------------------------------------------------------- epilogue
+    const int q = warp & 3;                      // TMEM lane quadrant this warp may read
+    const uint32_t tmem_empty_leader = mapa(tmem_empty, 0);
+    uint32_t tcount = 0;
+    const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15u) == 0) && (p.ldc % 4 == 0);
+    for (int t = pair; t < p.total_tiles; t += num_pairs, ++tcount) {
+      const PairTile tc = pair_tile(p, t);
+      const uint32_t acc = tcount & 1u, aph = (tcount >> 1) & 1u;
+      if (!mbar_wait(tmem_full + 8 * acc, aph, abort_flag)) break;
+      tc_fence_after();
+      const int64_t row = static_cast<int64_t>(tc.m0) + rank * kRows + q * 32 + lane;
+      const bool row_ok = row < p.M;
+      float* crow = p.C + row * p.ldc + tc.n0;
+#pragma unroll 1
+      for (int c = 0; c < kPairN / 32; ++c) {
+        uint32_t r[32];
+        tc_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kPairN + c * 32, r);
+        tc_wait_ld();
+        const int64_t col0 = static_cast<int64_t>(tc.n0) + c * 32;
+        if (row_ok && col0 < p.N) {
+          if (vec_ok && col0 + 32 <= p.N) {
+#pragma unroll
+            for (int v = 0; v < 8; ++v)
+              *reinterpret_cast<uint4*>(crow + c * 32 + 4 * v) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+          } else {
+#pragma unroll
+            for (int v = 0; v < 32; ++v)
+              if (col0 + v < p.N) crow[c * 32 + v] = __uint_as_float(r[v]);
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive_cluster(tmem_empty_leader + 8 * acc);
+    }
+  } else {
+    // ---------------------------------------------------------------- decode
+    const int d = threadIdx.x - kDecodeWarp0 * 32;            // 0..511
+    const int h = d >> 8;                                     // which unit pair of the raw chunk
+    const int row = d & 255;                                  // 0..127 A rows, 128..255 B rows
+    const uint32_t r7 = static_cast<uint32_t>(row) & 7u;
+    // bytes [0, 80) of the row chunk hold units 0 and 1, bytes [64, 144) units 2 and 3
+    const uint32_t raw_row = static_cast<uint32_t>(row) * kRawRowBytes + static_cast<uint32_t>(h) * 64u;
+    const uint32_t dec_row = dec_base + static_cast<uint32_t>(2 * h) * kDecStageBytes + static_cast<uint32_t>(row) * 128u;
+    const uint32_t dec_empty0 = dec_empty + 16 * h;
+    const uint32_t dec_full0_leader = mapa(dec_full, 0) + 16 * h;
+    uint32_t n = 0;
+    bool ok = true;
+    for (int t = pair; t < p.total_tiles && ok; t += num_pairs) {
+      for (int kc = 0; kc < p.num_kc && ok; ++kc, ++n) {
+        const uint32_t s = n & 1u, ph = (n >> 1) & 1u;
+        if (!(ok = mbar_wait(raw_full + 8 * s, ph, abort_flag))) break;
+        uint32_t L[20];
+        const uint32_t src = raw_base + s * kRawStageBytes + raw_row;
+#pragma unroll
+        for (int i = 0; i < 5; ++i) {
+          const uint4 v = lds128(src + 16 * i);
+          L[4 * i] = v.x; L[4 * i + 1] = v.y; L[4 * i + 2] = v.z; L[4 * i + 3] = v.w;
+        }
+        // The stage is refilled through the async proxy (TMA) while it was read through the generic
+        // proxy: the proxy fence orders these reads before the release.
+        fence_proxy_async_smem();
+        mbar_arrive(raw_empty + 8 * s);
+        if (h == 0) ok = decode_two_units<0>(L, dec_row, r7, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
+        else ok = decode_two_units<2>(L, dec_row, r7, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncwarp();
+  if (*abort_flag) {
+    // Some wait gave up: give copies and MMAs that are still in flight time to land before the
+    // shared and tensor memory they target is released.
+    const uint64_t t0 = global_ns();
+    while (global_ns() - t0 < 2000000ull) {}
+    if (threadIdx.x == 0) atomicExch(p.error_word, 1u);
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();            // neither CTA leaves while the other may still read its shared memory or arrive on its barriers
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+}  // namespace
+
+bool gemm_tc2_supported(const void* A, const void* B, int64_t M, int64_t N, int64_t K) {
+  if (!gemm_tc_supported(A, B, M, N, N, K)) return false;
+  return M < (1ll << 31) - kPairM && N < (1ll << 31) - kPairN && sm_count() >= 2;
+}
+
+hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,
+                            cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+      return HIF4_ERR_CUDA;
+    attr_set = true;
+  }
+  CUtensorMap tmA, tmB;
+  const int64_t upr = K / kUnitElems;
+  if (!make_unit_map(&tmA, A, M, upr, kRows) || !make_unit_map(&tmB, B, N, upr, kRows)) return HIF4_ERR_CUDA;
+  Gemm2Params p{};
+  p.C = C; p.ldc = ldc; p.M = M; p.N = N;
+  p.num_kc = static_cast<int>(K / (kRawUnits * kUnitElems));
+  p.n_tiles = static_cast<int>(ceil_div64(N, kPairN));
+  const int64_t tiles = ceil_div64(M, kPairM) * p.n_tiles;
+  if (tiles > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
+  p.total_tiles = static_cast<int>(tiles);
+  p.error_word = device_error_word();
+  if (!p.error_word) return HIF4_ERR_CUDA;
+  const int pairs = static_cast<int>(tiles < sm_count() / 2 ? tiles : sm_count() / 2);
+  gemm_tc2_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tmA, tmB, p);
+  note_launch();
+  return launch_status();
+}
+
+}  // namespace hif4

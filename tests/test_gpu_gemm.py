@@ -145,16 +145,18 @@ def test_grouped_gemm_moe_routing_sampled(hif4):
 
 
 # ------------------------------------------------------------------ tensor-core (tcgen05) kernel
-@pytest.fixture()
-def tc_path(hif4):
-    hif4.hif4_set_gemm_path(2)
+@pytest.fixture(params=[2, 3], ids=["one_cta", "cta_pair"])
+def tc_path(hif4, request):
+    """2 = single-CTA 128 x 256 kernel, 3 = CTA-pair 256 x 256 kernel, forced whatever the shape."""
+    hif4.hif4_set_gemm_path(request.param)
     yield hif4
     hif4.hif4_set_gemm_path(0)
     assert hif4.hif4_last_device_status() == 0, "a bounded wait inside the kernel ran out"
 
 
 @pytest.mark.parametrize("M,N,K", [(128, 256, 256), (128, 256, 512), (1, 64, 256), (130, 257, 768), (300, 700, 1024),
-                                   (64, 2000, 256), (1000, 130, 2048)])
+                                   (64, 2000, 256), (1000, 130, 2048), (256, 256, 256), (513, 385, 512),
+                                   (2500, 1300, 1280)])
 def test_tensor_core_kernel_full_compare(tc_path, M, N, K):
     hif4 = tc_path
     g = torch.Generator(device="cuda"); g.manual_seed(M * 7 + N)
