@@ -72,8 +72,11 @@ __device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
   return r;
 }
+// Arrive on a barrier of another CTA of the cluster.  The data this signals was written to shared
+// memory and ordered by fence.proxy.async before the call; a release at cluster scope on top of that
+// costs a full memory barrier per call and buys nothing for shared-memory data.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -135,10 +138,14 @@ __device__ __forceinline__ bool decode_two_units(const uint32_t (&L)[20], uint32
                                                  volatile uint32_t* abort_flag) {
 #pragma unroll
   for (int u = 0; u < 2; ++u) {
-    if (!mbar_wait(dec_empty0 + 8 * u, parity_free, abort_flag)) return false;
+    // warp-uniform outcome, so that the warp barrier below is never reached by a part of the warp
+    if (!__all_sync(0xFFFFFFFFu, mbar_wait(dec_empty0 + 8 * u, parity_free, abort_flag))) return false;
     decode_unit_to_row(L[kOff + 9 * u], &L[kOff + 9 * u + 1], stage0_row_addr + u * kDecStageBytes, r7);
     fence_proxy_async_smem();                  // generic-proxy writes -> visible to the tensor core
-    mbar_arrive_cluster(dec_full0_leader + 8 * u);
+    // One remote arrive per warp; the warp barrier orders the other lanes' writes and proxy fences
+    // before it.
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive_cluster(dec_full0_leader + 8 * u);
   }
   return true;
 }
@@ -168,12 +175,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       mbar_init(raw_empty + 8 * s, kDecodeThreads);
     }
     for (int s = 0; s < kDecStages; ++s) {
-      mbar_init(dec_full + 8 * s, kDecodeThreads);    // 256 threads of each CTA per stage (used on rank 0)
+      mbar_init(dec_full + 8 * s, kDecodeThreads / 32);   // 8 warps of each CTA per stage (used on rank 0)
       mbar_init(dec_empty + 8 * s, 1);
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(tmem_full + 8 * s, 1);
-      mbar_init(tmem_empty + 8 * s, 256);             // 128 epilogue threads of each CTA (used on rank 0)
+      mbar_init(tmem_empty + 8 * s, 8);               // 4 epilogue warps of each CTA (used on rank 0)
     }
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -244,7 +251,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     for (int t = pair; t < p.total_tiles; t += num_pairs, ++tcount) {
       const PairTile tc = pair_tile(p, t);
       const uint32_t acc = tcount & 1u, aph = (tcount >> 1) & 1u;
-      if (!mbar_wait(tmem_full + 8 * acc, aph, abort_flag)) break;
+      if (!__all_sync(0xFFFFFFFFu, mbar_wait(tmem_full + 8 * acc, aph, abort_flag))) break;
       tc_fence_after();
       const int64_t row = static_cast<int64_t>(tc.m0) + rank * kRows + q * 32 + lane;
       const bool row_ok = row < p.M;
@@ -268,7 +275,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
       }
       tc_fence_before();
-      mbar_arrive_cluster(tmem_empty_leader + 8 * acc);
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + 8 * acc);
     }
   } else {
     // ---------------------------------------------------------------- decode
@@ -286,7 +294,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     for (int t = pair; t < p.total_tiles && ok; t += num_pairs) {
       for (int kc = 0; kc < p.num_kc && ok; ++kc, ++n) {
         const uint32_t s = n & 1u, ph = (n >> 1) & 1u;
-        if (!(ok = mbar_wait(raw_full + 8 * s, ph, abort_flag))) break;
+        if (!(ok = __all_sync(0xFFFFFFFFu, mbar_wait(raw_full + 8 * s, ph, abort_flag)))) break;
         uint32_t L[20];
         const uint32_t src = raw_base + s * kRawStageBytes + raw_row;
 #pragma unroll
