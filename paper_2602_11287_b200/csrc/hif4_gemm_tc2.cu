@@ -43,7 +43,8 @@ constexpr int kDecodeWarp0 = 6;
 constexpr int kDecodeThreads = 4 * kRows;             // 512: (A rows + B rows) x 2 unit pairs
 constexpr int kThreads = kDecodeWarp0 * 32 + kDecodeThreads;   // 704
 
-constexpr int kSmemBytes = 1024 /*alignment slack*/ + kDecStages * kDecStageBytes + kRawStages * kRawStageBytes + 256;
+constexpr int kSmemBytes = 1024 /*alignment slack*/ + kDecStages * kDecStageBytes + kRawStages * kRawStageBytes + 256 +
+                           1024 /*spread table*/;
 
 // tcgen05.mma kind::f16 instruction descriptor: D = F32, A = B = BF16, both K-major, N/8, M/16.
 constexpr uint32_t kInstrDesc2 = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kPairN >> 3) << 17) |
@@ -58,6 +59,7 @@ struct Gemm2Params {
   int n_tiles;          // ceil(N / 256)
   int total_tiles;
   unsigned int* error_word;
+  DecodeMul mul;
 };
 
 // ------------------------------------------------------------------------------ cluster-scope PTX
@@ -133,14 +135,14 @@ __device__ __forceinline__ PairTile pair_tile(const Gemm2Params& p, int t) {
 // Decodes the two units held in raw words L[kOff .. kOff+8] and L[kOff+9 .. kOff+17] into decoded
 // stages 2h and 2h+1.  Returns false when a wait gave up.
 template <int kOff>
-__device__ __forceinline__ bool decode_two_units(const uint32_t (&L)[20], uint32_t stage0_row_addr, uint32_t r7,
-                                                 uint32_t dec_empty0, uint32_t dec_full0_leader, uint32_t parity_free,
-                                                 volatile uint32_t* abort_flag) {
+__device__ __forceinline__ bool decode_two_units(const uint32_t (&L)[20], const uint32_t (&chunk_addr)[8], uint32_t lut,
+                                                 const DecodeMul& mul, uint32_t dec_empty0, uint32_t dec_full0_leader,
+                                                 uint32_t parity_free, volatile uint32_t* abort_flag) {
 #pragma unroll
   for (int u = 0; u < 2; ++u) {
     // warp-uniform outcome, so that the warp barrier below is never reached by a part of the warp
     if (!__all_sync(0xFFFFFFFFu, mbar_wait(dec_empty0 + 8 * u, parity_free, abort_flag))) return false;
-    decode_unit_to_row(L[kOff + 9 * u], &L[kOff + 9 * u + 1], stage0_row_addr + u * kDecStageBytes, r7);
+    decode_unit_balanced(L[kOff + 9 * u], &L[kOff + 9 * u + 1], chunk_addr, u * kDecStageBytes, lut, mul);
     fence_proxy_async_smem();                  // generic-proxy writes -> visible to the tensor core
     // One remote arrive per warp; the warp barrier orders the other lanes' writes and proxy fences
     // before it.
@@ -164,6 +166,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
   volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(gen_base + (bar_base - smem_base) + 128);
   volatile uint32_t* abort_flag = tmem_ptr_smem + 1;
+  const uint32_t lut = bar_base + 256;
+  if (threadIdx.x < 256)
+    reinterpret_cast<uint32_t*>(gen_base + (lut - smem_base))[threadIdx.x] = spread_e8_entry(threadIdx.x);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
@@ -226,15 +231,18 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * kPairN;
         for (int kc = 0; kc < p.num_kc && ok; ++kc, ++n) {
+          // The two halves of the decode threads fill stages (0, 1) and (2, 3) side by side, so stages
+          // 0 and 2 are ready first: the K blocks of a chunk are consumed in the order 0, 2, 1, 3.
 #pragma unroll
-          for (int u = 0; u < kDecStages; ++u) {
+          for (int i = 0; i < kDecStages; ++i) {
+            const int u = ((i & 1) << 1) | (i >> 1);
             if (!(ok = mbar_wait_cluster(dec_full + 8 * u, n & 1u, abort_flag))) break;
             tc_fence_after();
             const uint64_t adesc = make_desc(dec_base + u * kDecStageBytes);
             const uint64_t bdesc = make_desc(dec_base + u * kDecStageBytes + kDecHalfBytes);
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-              tc2_mma(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, kInstrDesc2, (kc | u | kk) != 0 ? 1u : 0u);
+              tc2_mma(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, kInstrDesc2, (kc | i | kk) != 0 ? 1u : 0u);
             tc2_commit_both(dec_empty + 8 * u);       // both CTAs may overwrite the stage once these MMAs have read it
           }
         }
@@ -287,6 +295,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     // bytes [0, 80) of the row chunk hold units 0 and 1, bytes [64, 144) units 2 and 3
     const uint32_t raw_row = static_cast<uint32_t>(row) * kRawRowBytes + static_cast<uint32_t>(h) * 64u;
     const uint32_t dec_row = dec_base + static_cast<uint32_t>(2 * h) * kDecStageBytes + static_cast<uint32_t>(row) * 128u;
+    uint32_t chunk_addr[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) chunk_addr[j] = dec_row + ((static_cast<uint32_t>(j) ^ r7) << 4);
     const uint32_t dec_empty0 = dec_empty + 16 * h;
     const uint32_t dec_full0_leader = mapa(dec_full, 0) + 16 * h;
     uint32_t n = 0;
@@ -306,8 +317,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         // proxy: the proxy fence orders these reads before the release.
         fence_proxy_async_smem();
         mbar_arrive(raw_empty + 8 * s);
-        if (h == 0) ok = decode_two_units<0>(L, dec_row, r7, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
-        else ok = decode_two_units<2>(L, dec_row, r7, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
+        if (h == 0) ok = decode_two_units<0>(L, chunk_addr, lut, p.mul, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
+        else ok = decode_two_units<2>(L, chunk_addr, lut, p.mul, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
       }
     }
   }
@@ -356,6 +367,7 @@ hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, i
   p.total_tiles = static_cast<int>(tiles);
   p.error_word = device_error_word();
   if (!p.error_word) return HIF4_ERR_CUDA;
+  p.mul = make_decode_mul();
   const int pairs = static_cast<int>(tiles < sm_count() / 2 ? tiles : sm_count() / 2);
   gemm_tc2_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tmA, tmB, p);
   note_launch();

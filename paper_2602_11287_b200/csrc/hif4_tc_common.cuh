@@ -144,6 +144,64 @@ __device__ __forceinline__ void decode_unit_to_row(uint32_t meta, const uint32_t
   }
 }
 
+// ---- pipe-balanced decoder
+// The decode is bound by instruction issue on the integer/logic pipe, while the pipe that runs integer
+// multiply-adds and packed BF16 FMAs is mostly idle.  This variant moves every left shift and most
+// additions onto that pipe by writing them as multiply-adds with multipliers that the compiler cannot
+// see (kernel parameters), takes the sum of the micro-exponents of all eight level-2 groups at once
+// (two-bit fields), and uses store addresses that are computed once per thread.
+struct DecodeMul {            // runtime-valued on purpose: 1, 2, 8, 16, 32, 128, 256, 4096
+  uint32_t one, m2, m8, m16, m32, m128, m256, m4096;
+};
+inline DecodeMul make_decode_mul() { return DecodeMul{1u, 2u, 8u, 16u, 32u, 128u, 256u, 4096u}; }
+
+// 256-entry table in shared memory: bit i of the index spread to bit 2i, replicated in both halves.
+__device__ __forceinline__ uint32_t spread_e8_entry(uint32_t x) {
+  x = (x | (x << 4)) & 0x0F0Fu;
+  x = (x | (x << 2)) & 0x3333u;
+  x = (x | (x << 1)) & 0x5555u;
+  return x * 0x10001u;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+
+// Decodes one unit into one 128-byte operand row; chunk_addr[j] is the shared-memory address of the
+// 16-byte chunk that word j of this thread's row goes to (swizzle applied) inside stage 0, `stage_off`
+// the byte offset of the target stage, `lut` the address of the spread table.
+__device__ __forceinline__ void decode_unit_balanced(uint32_t meta, const uint32_t* w, const uint32_t (&chunk_addr)[8],
+                                                     uint32_t stage_off, uint32_t lut, const DecodeMul& k) {
+  const uint32_t byte = meta & 0xFFu;
+  if (byte == 0xFFu) {                           // NaN unit (Eq. 2): every element is NaN
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      sts128(chunk_addr[j] + stage_off, 0x7FC07FC0u, 0x7FC07FC0u, 0x7FC07FC0u, 0x7FC07FC0u);
+    return;
+  }
+  // BF16 bits of E6M2 / 4 in both halves: ((byte + 308) << 5) * 0x10001
+  const uint32_t base2 = byte * 0x00200020u + 0x26802680u;
+  // Two-bit fields: field j of the low half = E1_8[j] + E1_16[2j], of the high half = E1_8[j] + E1_16[2j+1]
+  const uint32_t sum = (((meta >> 16) & 0x5555u) | ((meta >> 1) & 0x55550000u)) + lds32(lut + ((meta >> 6) & 0x3FCu));
+  const uint32_t sumh = sum >> 8;
+  const uint32_t mul[4] = {k.m128, k.m32, k.m8, k.m2};
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const uint32_t f = ((j < 4 ? sum : sumh) * mul[j & 3]) & 0x01800180u;       // field j at the exponent's low bits
+    const uint32_t Sa = f * k.one + base2;                            // (S_lo, S_hi), S = E6M2 * 2^(e8 + e16 - 2)
+    const uint32_t Sb = Sa - 0x02000200u;                             // S / 16
+    const uint32_t Oa = Sa * k.one + 0x83808380u;                     // -128 S
+    const uint32_t Ob = Sa * k.one + 0x81808180u;                     // -8 S
+    const uint32_t wj = w[j], wh = wj >> 8;
+    const uint32_t r0 = fma_bf16x2((wj & 0x00070007u) | 0x43004300u, Sa, Oa) ^ ((wj * k.m4096) & 0x80008000u);  // elements 0, 4
+    const uint32_t r1 = fma_bf16x2((wj & 0x00700070u) | 0x43004300u, Sb, Ob) ^ ((wj * k.m256) & 0x80008000u);   // elements 1, 5
+    const uint32_t r2 = fma_bf16x2((wh & 0x00070007u) | 0x43004300u, Sa, Oa) ^ ((wj * k.m16) & 0x80008000u);    // elements 2, 6
+    const uint32_t r3 = fma_bf16x2((wh & 0x00700070u) | 0x43004300u, Sb, Ob) ^ (wj & 0x80008000u);              // elements 3, 7
+    sts128(chunk_addr[j] + stage_off, r0, r1, r2, r3);
+  }
+}
+
 // ------------------------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
