@@ -14,7 +14,9 @@
 //   warp 1       rank 0 only: issues tcgen05.mma.cta_group::2 (256 x 256 x 16, four per K block), which
 //                reads A and B halves from both CTAs' shared memory and accumulates into both CTAs'
 //                tensor memory; commits are multicast to the barriers of both CTAs
-//   warps 2-5    epilogue: tcgen05.ld of this CTA's 128 accumulator rows, FP32 stores to C
+//   warps 2-5    epilogue: tcgen05.ld of this CTA's 128 accumulator rows, 32 x 16 FP32 slabs staged in
+//                shared memory (SWIZZLE_64B) and written to C with TMA stores, which also clip the
+//                ragged edges; plain per-thread stores when C is not 16-byte aligned
 // Cross-CTA signalling: "decoded stage full" and "accumulator drained" are mbarriers of rank 0 on which
 // the threads of both CTAs arrive (remote arrives with release at cluster scope); "stage free" and
 // "accumulator complete" arrive in both CTAs through the multicast commit.
@@ -43,8 +45,11 @@ constexpr int kDecodeWarp0 = 6;
 constexpr int kDecodeThreads = 4 * kRows;             // 512: (A rows + B rows) x 2 unit pairs
 constexpr int kThreads = kDecodeWarp0 * 32 + kDecodeThreads;   // 704
 
-constexpr int kSmemBytes = 1024 /*alignment slack*/ + kDecStages * kDecStageBytes + kRawStages * kRawStageBytes + 256 +
-                           1024 /*spread table*/;
+constexpr int kEpiCols = 16;                          // FP32 columns per staged slab (64-byte rows)
+constexpr int kEpiSlabBytes = 32 * kEpiCols * 4;      // 32 rows of one epilogue warp: 2048
+constexpr int kEpiBytes = 4 * 2 * kEpiSlabBytes;      // 4 warps x 2 buffers
+constexpr int kSmemBytes = 1024 /*alignment slack*/ + kDecStages * kDecStageBytes + kRawStages * kRawStageBytes + kEpiBytes +
+                           256 /*barriers*/ + 1024 /*spread table*/;
 
 // tcgen05.mma kind::f16 instruction descriptor: D = F32, A = B = BF16, both K-major, N/8, M/16.
 constexpr uint32_t kInstrDesc2 = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kPairN >> 3) << 17) |
@@ -59,6 +64,7 @@ struct Gemm2Params {
   int n_tiles;          // ceil(N / 256)
   int total_tiles;
   unsigned int* error_word;
+  int tma_store;        // 1: C goes out through the tensor map tmC, 0: per-thread stores
   DecodeMul mul;
 };
 
@@ -126,6 +132,28 @@ __device__ __forceinline__ void tc2_mma(uint32_t d_tmem, uint64_t adesc, uint64_
       : "memory");
 }
 
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(x),
+               "r"(y), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Waits until all but the newest `kPending` bulk groups of this thread have finished reading shared memory.
+template <int kPending>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kPending) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 struct PairTile { int m0; int n0; };
 __device__ __forceinline__ PairTile pair_tile(const Gemm2Params& p, int t) {
   const int mt = t / p.n_tiles;
@@ -154,12 +182,13 @@ __device__ __forceinline__ bool decode_two_units(const uint32_t (&L)[20], const 
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                const Gemm2Params p) {
+                const __grid_constant__ CUtensorMap tmC, const Gemm2Params p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t dec_base = smem_base;                                        // 1024-byte aligned stages
   const uint32_t raw_base = dec_base + kDecStages * kDecStageBytes;
-  const uint32_t bar_base = raw_base + kRawStages * kRawStageBytes;
+  const uint32_t epi_base = raw_base + kRawStages * kRawStageBytes;          // 1024-byte aligned as well
+  const uint32_t bar_base = epi_base + kEpiBytes;
   // barriers (8 bytes each)
   const uint32_t raw_full = bar_base, raw_empty = bar_base + 16, dec_full = bar_base + 32, dec_empty = bar_base + 64,
                  tmem_full = bar_base + 96, tmem_empty = bar_base + 112;
@@ -211,7 +240,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const PairTile tc = pair_tile(p, t);
         for (int kc = 0; kc < p.num_kc; ++kc, ++n) {
           const uint32_t s = n & 1u, ph = (n >> 1) & 1u;
-          if (!(ok = mbar_wait(raw_empty + 8 * s, ph ^ 1u, abort_flag))) break;
+          if (!(ok = mbar_wait(raw_empty + 8 * s, ph ^ 1u, abort_flag, 128))) break;
           mbar_expect_tx(raw_full + 8 * s, kRawStageBytes);
           const uint32_t dst = raw_base + s * kRawStageBytes;
           tma_load_2d(dst, &tmA, kc * kRawRowBytes, tc.m0 + static_cast<int>(rank) * kRows, raw_full + 8 * s);
@@ -255,36 +284,76 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int q = warp & 3;                      // TMEM lane quadrant this warp may read
     const uint32_t tmem_empty_leader = mapa(tmem_empty, 0);
     uint32_t tcount = 0;
-    const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15u) == 0) && (p.ldc % 4 == 0);
-    for (int t = pair; t < p.total_tiles; t += num_pairs, ++tcount) {
-      const PairTile tc = pair_tile(p, t);
-      const uint32_t acc = tcount & 1u, aph = (tcount >> 1) & 1u;
-      if (!__all_sync(0xFFFFFFFFu, mbar_wait(tmem_full + 8 * acc, aph, abort_flag))) break;
-      tc_fence_after();
-      const int64_t row = static_cast<int64_t>(tc.m0) + rank * kRows + q * 32 + lane;
-      const bool row_ok = row < p.M;
-      float* crow = p.C + row * p.ldc + tc.n0;
+    if (p.tma_store) {
+      // Slab = this warp's 32 rows x 16 columns, 64-byte rows, 16-byte chunk c of row r stored at chunk
+      // c ^ ((r >> 1) & 3) (SWIZZLE_64B): conflict-free 128-bit stores, and the TMA store undoes it.
+      const uint32_t slab0 = epi_base + static_cast<uint32_t>(q) * (2 * kEpiSlabBytes);
+      const uint32_t my_row = slab0 + static_cast<uint32_t>(lane) * 64u;
+      const uint32_t sw = (static_cast<uint32_t>(lane) >> 1) & 3u;
+      uint32_t slabs = 0;
+      for (int t = pair; t < p.total_tiles; t += num_pairs, ++tcount) {
+        const PairTile tc = pair_tile(p, t);
+        const uint32_t acc = tcount & 1u, aph = (tcount >> 1) & 1u;
+        if (!__all_sync(0xFFFFFFFFu, mbar_wait(tmem_full + 8 * acc, aph, abort_flag, 256))) break;
+        tc_fence_after();
+        const int row0 = tc.m0 + static_cast<int>(rank) * kRows + q * 32;
 #pragma unroll 1
-      for (int c = 0; c < kPairN / 32; ++c) {
-        uint32_t r[32];
-        tc_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kPairN + c * 32, r);
-        tc_wait_ld();
-        const int64_t col0 = static_cast<int64_t>(tc.n0) + c * 32;
-        if (row_ok && col0 < p.N) {
-          if (vec_ok && col0 + 32 <= p.N) {
+        for (int c = 0; c < kPairN / kEpiCols; ++c, ++slabs) {
+          uint32_t r[16];
+          tc_ld16(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kPairN + c * kEpiCols, r);
+          tc_wait_ld();
+          if (c == kPairN / kEpiCols - 1) {          // accumulator fully read: hand it back before the stores
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + 8 * acc);
+          }
+          const uint32_t buf = (slabs & 1u) * kEpiSlabBytes;
+          if (lane == 0) bulk_wait_read<1>();        // the store that used this buffer two slabs ago has read it
+          __syncwarp();
 #pragma unroll
-            for (int v = 0; v < 8; ++v)
-              *reinterpret_cast<uint4*>(crow + c * 32 + 4 * v) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
-          } else {
-#pragma unroll
-            for (int v = 0; v < 32; ++v)
-              if (col0 + v < p.N) crow[c * 32 + v] = __uint_as_float(r[v]);
+          for (int v = 0; v < 4; ++v)
+            sts128(my_row + buf + ((static_cast<uint32_t>(v) ^ sw) << 4), r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+          fence_proxy_async_smem();                  // generic-proxy writes -> visible to the TMA store
+          __syncwarp();
+          if (lane == 0 && row0 < p.M && tc.n0 + c * kEpiCols < p.N) {
+            tma_store_2d(&tmC, tc.n0 + c * kEpiCols, row0, slab0 + buf);
+            bulk_commit();
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + 8 * acc);
+      if (lane == 0) bulk_wait_all();                // shared memory stays valid until the last store has read it
+    } else {
+      const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15u) == 0) && (p.ldc % 4 == 0);
+      for (int t = pair; t < p.total_tiles; t += num_pairs, ++tcount) {
+        const PairTile tc = pair_tile(p, t);
+        const uint32_t acc = tcount & 1u, aph = (tcount >> 1) & 1u;
+        if (!__all_sync(0xFFFFFFFFu, mbar_wait(tmem_full + 8 * acc, aph, abort_flag, 256))) break;
+        tc_fence_after();
+        const int64_t row = static_cast<int64_t>(tc.m0) + rank * kRows + q * 32 + lane;
+        const bool row_ok = row < p.M;
+        float* crow = p.C + row * p.ldc + tc.n0;
+#pragma unroll 1
+        for (int c = 0; c < kPairN / 32; ++c) {
+          uint32_t r[32];
+          tc_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kPairN + c * 32, r);
+          tc_wait_ld();
+          const int64_t col0 = static_cast<int64_t>(tc.n0) + c * 32;
+          if (row_ok && col0 < p.N) {
+            if (vec_ok && col0 + 32 <= p.N) {
+#pragma unroll
+              for (int v = 0; v < 8; ++v)
+                *reinterpret_cast<uint4*>(crow + c * 32 + 4 * v) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+            } else {
+#pragma unroll
+              for (int v = 0; v < 32; ++v)
+                if (col0 + v < p.N) crow[c * 32 + v] = __uint_as_float(r[v]);
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + 8 * acc);
+      }
     }
   } else {
     // ---------------------------------------------------------------- decode
@@ -340,6 +409,18 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   }
 }
 
+// FP32 view of C for the TMA stores of the epilogue: box = 16 columns x 32 rows, SWIZZLE_64B.
+bool make_c_map(CUtensorMap* map, float* C, int64_t M, int64_t N, int64_t ldc) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(M)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ldc) * 4};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kEpiCols), 32};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 bool gemm_tc2_supported(const void* A, const void* B, int64_t M, int64_t N, int64_t K) {
@@ -368,8 +449,10 @@ hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, i
   p.error_word = device_error_word();
   if (!p.error_word) return HIF4_ERR_CUDA;
   p.mul = make_decode_mul();
+  CUtensorMap tmC = tmA;                              // placeholder when the store path is not used
+  p.tma_store = ((reinterpret_cast<uintptr_t>(C) & 15u) == 0 && ldc % 4 == 0 && make_c_map(&tmC, C, M, N, ldc)) ? 1 : 0;
   const int pairs = static_cast<int>(tiles < sm_count() / 2 ? tiles : sm_count() / 2);
-  gemm_tc2_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tmA, tmB, p);
+  gemm_tc2_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tmA, tmB, tmC, p);
   note_launch();
   return launch_status();
 }

@@ -45,11 +45,15 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false when the budget ran out or another thread has already given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+// Roles that wait long (a whole tile, a whole raw chunk) pass `sleep_ns` > 0 and back off between
+// polls, so that their spinning does not take issue slots from the decode warps.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t sleep_ns = 0) {
   if (mbar_try(bar, parity)) return true;
   const uint64_t t0 = global_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try(bar, parity)) return true;
+    if (sleep_ns) __nanosleep(sleep_ns);
     if ((it & 63u) == 0u) {
       if (*abort_flag) return false;
       if (global_ns() - t0 > kWaitBudgetNs) {

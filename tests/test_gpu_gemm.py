@@ -190,6 +190,18 @@ def test_tensor_core_kernel_random_units_nan_and_guard_bands(tc_path):
     assert (out[0] == -5.0).all() and (out[M + 1] == -5.0).all() and (out[:, N:] == -5.0).all()
 
 
+def test_tensor_core_kernel_c_rows_not_16_byte_aligned(tc_path):
+    """ldc odd and a base that is only 4-byte aligned: the kernels fall back from vector / TMA stores."""
+    hif4 = tc_path
+    M, N, K = 300, 333, 512
+    g = torch.Generator(device="cuda"); g.manual_seed(77)
+    a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
+    b = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
+    buf = torch.full((M + 2, N + 2), -5.0, dtype=torch.float32, device="cuda")
+    check_full(hif4, a, b, "unaligned C", out=buf[1:M + 1, 1:N + 1])
+    assert (buf[0] == -5.0).all() and (buf[M + 1] == -5.0).all() and (buf[:, 0] == -5.0).all() and (buf[:, N + 1] == -5.0).all()
+
+
 def test_tensor_core_grouped(tc_path):
     hif4 = tc_path
     _grouped_case(hif4, [3, 0, 70, 1, 0, 129, 64, 0, 300], N=300, K=256, seed=61)
