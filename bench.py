@@ -395,14 +395,15 @@ def run_case(spec: str):
     nums = [int(v) for v in rest.split(",") if v]
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
-    reps = 5
+    reps = 20
     if kind == "gemm":
         M, N, K = nums
         a = hif4.hif4_quantize(wl.llama_activations(M, K, device=dev))
         b = hif4.hif4_quantize(wl.gaussian(N, K, 0.02, seed=5, device=dev))
         c = torch.empty(M, N, dtype=torch.float32, device=dev)
-        fn = lambda: hif4.hif4_gemm(a, b, out=c)
-        work = f"{flops(M, K, N) / 1e9:.1f} GFLOP"
+        ws = torch.empty(max(hif4.hif4_gemm_workspace(M, N, K), 256), dtype=torch.uint8, device=dev)
+        fn = lambda: hif4.hif4_gemm(a, b, out=c, workspace=ws)
+        work = f"{flops(M, K, N) / 1e9:.1f} GFLOP, min traffic {gemm_min_bytes(M, K, N) / 1e6:.1f} MB"
     elif kind in ("quantize", "dequantize"):
         n = 2 ** nums[0]
         x = wl.quantize_sweep(n, device=dev)
@@ -425,6 +426,7 @@ def run_case(spec: str):
     fn()
     torch.cuda.synchronize()
     s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda._sleep(4_000_000)          # keeps the GPU busy while the host queues the launches below
     s.record()
     for _ in range(reps):
         fn()

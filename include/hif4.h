@@ -90,7 +90,8 @@ hif4_status hif4_quantize(const void* src, hif4_dtype dt, int64_t rows, int64_t 
 hif4_status hif4_dequantize(const void* src_units, int64_t rows, int64_t cols, void* dst,
                             hif4_dtype dt, int64_t ld_dst, void* stream);
 
-/* Workspace (device scratch) that hif4_gemm needs for this shape; may be 0.  Host-only.  */
+/* Workspace (device scratch) that hif4_gemm needs for this shape; may be 0 (for M <= 16 it holds
+ * the decoded activation rows: 2 * K * 8 or 16 bytes).  Host-only.  */
 hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size_t* bytes);
 
 /* hif4_gemm -- C = A * B^T with A, B in HiF4 and FP32 accumulation: C[i][j] is the sum over the
@@ -165,7 +166,8 @@ const char* hif4_status_string(hif4_status s);
 /* Diagnostic: 0 = choose the GEMM kernel by shape (default), 1 = CUDA-core kernel only, 2 = the
  * single-CTA tensor-core (tcgen05) kernel whenever it is legal (K % 256 == 0, 16-byte aligned
  * operands), even for small M, 3 = the CTA-pair tensor-core kernel (256 x 256 tiles) whenever it is
- * legal.  Process-wide, not thread-safe; meant for tests and benchmarks.  */
+ * legal, 4 = the weight-streaming kernel whenever it is legal (M <= 16).  Process-wide, not
+ * thread-safe; meant for tests and benchmarks.  */
 hif4_status hif4_set_gemm_path(int path);
 
 /* Number of kernels this library has launched in this process (monotonic, host-side counter).  */

@@ -6,9 +6,9 @@ using namespace hif4;
 
 namespace {
 // 0 = choose by shape, 1 = CUDA-core kernel only, 2 = single-CTA tensor-core kernel whenever it is
-// legal, 3 = CTA-pair tensor-core kernel whenever it is legal.
+// legal, 3 = CTA-pair tensor-core kernel whenever it is legal, 4 = weight-streaming kernel whenever
+// it is legal (M <= 16).
 int g_gemm_path = 0;
-constexpr int64_t kTensorCoreMinM = 64;
 constexpr int64_t kPairMinM = 129;      // below that a 256-row pair tile would be half empty
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -26,12 +26,12 @@ hif4_status check_common(const void* A, const void* B, const float* C, int64_t M
 extern "C" hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size_t* bytes) {
   if (!bytes) return HIF4_ERR_NULL;
   if (M < 0 || N < 0 || K < 0 || K % kUnitElems != 0) return HIF4_ERR_SHAPE;
-  *bytes = 0;
+  *bytes = gemv_workspace_bytes(M, K);       // decoded tokens of the weight-streaming path (M <= 16)
   return HIF4_OK;
 }
 
 extern "C" hif4_status hif4_set_gemm_path(int path) {
-  if (path < 0 || path > 3) return HIF4_ERR_DTYPE;
+  if (path < 0 || path > 4) return HIF4_ERR_DTYPE;
   g_gemm_path = path;
   return HIF4_OK;
 }
@@ -39,8 +39,6 @@ extern "C" hif4_status hif4_set_gemm_path(int path) {
 extern "C" hif4_status hif4_gemm(const void* A_units, const void* B_units, float* C, int64_t M, int64_t N,
                                  int64_t K, int64_t ldc, void* workspace, size_t workspace_bytes,
                                  void* stream) {
-  (void)workspace;
-  (void)workspace_bytes;
   const hif4_status chk = check_common(A_units, B_units, C, M, N, K, ldc);
   if (chk != HIF4_OK || M == 0 || N == 0) return chk;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -50,10 +48,15 @@ extern "C" hif4_status hif4_gemm(const void* A_units, const void* B_units, float
       return HIF4_ERR_CUDA;
     return HIF4_OK;
   }
+  if ((g_gemm_path == 0 || g_gemm_path == 4) && gemv_supported(A_units, B_units, M, N, K)) {
+    if (!workspace || workspace_bytes < gemv_workspace_bytes(M, K)) return HIF4_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return HIF4_ERR_ALIGN;
+    return launch_gemv(A_units, B_units, C, M, N, K, ldc, workspace, st);
+  }
   const bool tc_ok = g_gemm_path != 1 && gemm_tc_supported(A_units, B_units, M, N, N, K);
   if (tc_ok && g_gemm_path != 2 && (g_gemm_path == 3 || M >= kPairMinM) && gemm_tc2_supported(A_units, B_units, M, N, K))
     return launch_gemm_tc2(A_units, B_units, C, M, N, K, ldc, st);
-  if (tc_ok && (g_gemm_path >= 2 || M >= kTensorCoreMinM)) return launch_gemm_tc(A_units, B_units, C, M, N, K, ldc, st);
+  if (tc_ok && (g_gemm_path >= 2 || M > kGemvMaxM)) return launch_gemm_tc(A_units, B_units, C, M, N, K, ldc, st);
   return launch_gemm_simt(A_units, B_units, C, M, N, K, ldc, st);
 }
 

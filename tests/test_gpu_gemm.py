@@ -215,3 +215,58 @@ def test_tensor_core_prefill_shape_sampled(tc_path):
     w = hif4.hif4_quantize(wl.gaussian(N, K, 0.02, seed=71, device="cuda"))
     x = hif4.hif4_quantize(wl.llama_activations(M, K, device="cuda"))
     check_sampled(hif4, x, w, "tc llama qo M=4096", n=400)
+
+
+# ------------------------------------------------------------------ weight-streaming kernel (M <= 16)
+@pytest.fixture()
+def gemv_path(hif4):
+    hif4.hif4_set_gemm_path(4)
+    yield hif4
+    hif4.hif4_set_gemm_path(0)
+    assert hif4.hif4_last_device_status() == 0, "a bounded wait inside the kernel ran out"
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 1, 256), (1, 64, 256), (2, 33, 512), (7, 200, 1024), (8, 4096, 256), (9, 130, 768),
+                                   (16, 1000, 2304), (16, 64, 4096), (5, 9475, 256), (3, 31, 5120), (12, 77, 14336)])
+def test_weight_streaming_kernel_full_compare(gemv_path, M, N, K):
+    hif4 = gemv_path
+    g = torch.Generator(device="cuda"); g.manual_seed(M * 11 + N)
+    a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
+    b = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
+    assert hif4.hif4_gemm_workspace(M, N, K) == (8 if M <= 8 else 16) * K * 2
+    before = hif4.launch_count()
+    out = torch.full((M + 2, N + 3), -5.0, dtype=torch.float32, device="cuda")
+    C = check_full(hif4, a, b, f"gemv {M}x{N}x{K}", out=out[1:M + 1, 1:N + 1])
+    assert hif4.launch_count() - before == 2, "token preparation + streaming kernel"
+    assert (out[0] == -5.0).all() and (out[M + 1] == -5.0).all() and (out[:, 0] == -5.0).all() and (out[:, N + 1:] == -5.0).all()
+    C2 = hif4.hif4_gemm(a, b)
+    assert torch.equal(C.contiguous(), C2), "two runs of the weight-streaming kernel differ"
+
+
+def test_weight_streaming_kernel_random_units_and_nan(gemv_path):
+    hif4 = gemv_path
+    rng = np.random.default_rng(81)
+    M, N, upr = 11, 150, 8
+    A = rng.integers(0, 256, (M, upr, 36), dtype=np.uint8)
+    B = rng.integers(0, 256, (N, upr, 36), dtype=np.uint8)
+    A[..., 0] = rng.integers(0x00, 0xFF, (M, upr)); B[..., 0] = rng.integers(0x40, 0xC0, (N, upr))
+    A[3, 5, 0] = 0xFF
+    B[149, 0, 0] = 0xFF
+    C = hif4.hif4_gemm(torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda())
+    ref, refabs = oracle.gemm_f64(A, B, nthreads=8)
+    got = C.cpu().numpy().astype(np.float64)
+    nan = np.isnan(ref)
+    assert nan[3].all() and nan[:, 149].all() and np.array_equal(np.isnan(got), nan)
+    assert np.all(np.abs(got - ref)[~nan] <= TOL * refabs[~nan] + 1e-300)
+
+
+def test_weight_streaming_kernel_needs_its_workspace(gemv_path):
+    hif4 = gemv_path
+    a = torch.zeros(4, 4, 36, dtype=torch.uint8, device="cuda")
+    b = torch.zeros(64, 4, 36, dtype=torch.uint8, device="cuda")
+    c = torch.zeros(4, 64, dtype=torch.float32, device="cuda")
+    before = hif4.launch_count()
+    assert hif4.lib.hif4_gemm(a.data_ptr(), b.data_ptr(), c.data_ptr(), 4, 64, 256, 64, None, 0, None) == 5
+    ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    assert hif4.lib.hif4_gemm(a.data_ptr(), b.data_ptr(), c.data_ptr(), 4, 64, 256, 64, ws.data_ptr(), 1024, None) == 5
+    assert hif4.launch_count() == before
