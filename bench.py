@@ -119,9 +119,8 @@ def gemm_min_bytes(M, K, N):
 def run_cuda(args):
     import paper_2602_11287_b200 as hif4
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2602_11287_b200 import dp
+    rank, local_rank, world = dp.rank_info()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the HiF4 path has no CPU fallback")
     torch.cuda.set_device(local_rank)
@@ -140,7 +139,7 @@ def run_cuda(args):
     acts, xq, cs = {}, {}, {}
     for (M, K, N, name) in SHAPES:
         if (M, K) not in acts:
-            acts[(M, K)] = wl.llama_activations(M, K, seed=1002 + rank * 17 + M + K, device=dev)
+            acts[(M, K)] = wl.llama_activations(M, K, seed=dp.rank_seed(1002 + M + K, rank), device=dev)
         xq[(M, K, N)] = torch.empty(M, K // 64, 36, dtype=torch.uint8, device=dev)
         cs[(M, K, N)] = torch.empty(M, N, dtype=torch.float32, device=dev)
     # one scratch buffer for the GEMM workspaces (stream-ordered reuse)
@@ -163,9 +162,7 @@ def run_cuda(args):
                 events.append(((M, K, N), e0, e1, e2))
 
     def barrier():
-        if world > 1:
-            import torch.distributed as dist
-            dist.barrier()
+        dp.barrier()
         torch.cuda.synchronize()
 
     sampler = ClockSampler(local_rank)
@@ -187,19 +184,14 @@ def run_cuda(args):
     host_t1 = time.time()
     launches = hif4.launch_count() - launches0
     clocks = sampler.stop(host_t0, host_t1)
-    elapsed_ms = t_start.elapsed_time(t_end)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = dp.max_over_ranks(t_start.elapsed_time(t_end), dev)
     status = hif4.hif4_last_device_status()
     if status != 0:
         raise SystemExit(f"device status {status}: {hif4.status_string(status)}")
 
     step_flops = sum(flops(M, K, N) for (M, K, N, _) in SHAPES)
     ms_per_step = elapsed_ms / args.steps
-    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    value = dp.job_throughput(step_flops, world, ms_per_step * 1e-3) / 1e12
 
     # ---- per-kernel times inside the timed region
     per_shape = {}

@@ -1,0 +1,115 @@
+"""GPU parity at the full configured sizes, in the launch configuration bench.py times (default kernel
+selection).  The oracle cannot redo whole tensors of this size in seconds, so it recomputes sampled rows
+(quantizer: bit-exact) and sampled output entries plus the four corners (GEMM: the stated tolerance)."""
+import numpy as np
+import pytest
+import torch
+
+import hif4_workloads as wl
+import oracle
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def hif4():
+    assert torch.cuda.is_available()
+    import paper_2602_11287_b200 as lib
+    yield lib
+    assert lib.hif4_last_device_status() == 0
+    torch.cuda.empty_cache()
+
+
+def _sampled_rows_match(hif4, x, n_rows, seed):
+    q = hif4.hif4_quantize(x)
+    rng = np.random.default_rng(seed)
+    rows = np.unique(np.concatenate([rng.integers(0, x.shape[0], n_rows), [0, x.shape[0] - 1]]))
+    idx = torch.from_numpy(rows).cuda()
+    host = x[idx].cpu()
+    src = wl.bf16_to_u16_numpy(host) if x.dtype == torch.bfloat16 else host.numpy()
+    want = oracle.quantize(src, nthreads=8)
+    got = q[idx].cpu().numpy()
+    assert np.array_equal(got, want), f"{int((got != want).any(axis=-1).sum())} sampled units differ"
+    return q
+
+
+def test_quantize_sweep_sizes_sampled_rows(hif4):
+    """Config 3: 2^20 .. 2^28 BF16 elements of the Gaussian / Student-t / uniform mix with spike units."""
+    for log2n in (20, 24, 28):
+        x = wl.quantize_sweep(2 ** log2n, device="cuda")
+        q = _sampled_rows_match(hif4, x, 48, seed=log2n)
+        assert q.shape == (2 ** log2n // 4096, 64, 36)
+        del x, q
+    x32 = wl.quantize_sweep(2 ** 24, device="cuda", dtype=torch.float32)
+    _sampled_rows_match(hif4, x32, 48, seed=1)
+
+
+def _sampled_entries(hif4, a_units, b_units, C, what, n=300, seed=0):
+    M, N = C.shape
+    rng = np.random.default_rng(seed)
+    rows = np.concatenate([rng.integers(0, M, n), [0, M - 1, 0, M - 1]])
+    cols = np.concatenate([rng.integers(0, N, n), [0, 0, N - 1, N - 1]])
+    urows, rinv = np.unique(rows, return_inverse=True)
+    ucols, cinv = np.unique(cols, return_inverse=True)
+    a_host = a_units[torch.from_numpy(urows).cuda()].cpu().numpy()          # only the sampled rows travel to the host
+    b_host = b_units[torch.from_numpy(ucols).cuda()].cpu().numpy()
+    ref, refabs = oracle.gemm_sampled_f64(a_host, b_host, rinv, cinv)
+    got = C[torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()].cpu().numpy().astype(np.float64)
+    err = np.abs(got - ref)
+    assert np.all(err <= TOL * refabs + 1e-300), f"{what}: worst ratio {np.max(err / np.maximum(TOL * refabs, 1e-300)):.3g}"
+
+
+def test_llama_linears_all_m(hif4):
+    """Config 2 exactly as the benchmark runs it: every (M, K, N) through the default dispatch."""
+    for (name, K, N) in wl.LLAMA3_8B_LINEARS:
+        w = hif4.hif4_quantize(wl.gaussian(N, K, 0.02, seed=2000 + N + K, device="cuda"))
+        for M in wl.LLAMA3_8B_M:
+            x = hif4.hif4_quantize(wl.llama_activations(M, K, seed=1002 + M + K, device="cuda"))
+            C = hif4.hif4_gemm(x, w)
+            _sampled_entries(hif4, x, w, C, f"llama {name} M={M}", n=200, seed=M)
+            del C
+        del w
+
+
+def test_dense_prefill_m8192(hif4):
+    """Config 4: M = 8192 tokens with per-token scales over 2^-4 .. 2^4."""
+    for (name, K, N) in wl.DENSE_PREFILL_LINEARS:
+        x = hif4.hif4_quantize(wl.prefill_activations(wl.DENSE_PREFILL_M, K, device="cuda"))
+        w = hif4.hif4_quantize(wl.gaussian(N, K, 0.015, seed=4000 + N + K, device="cuda"))
+        C = hif4.hif4_gemm(x, w)
+        _sampled_entries(hif4, x, w, C, f"prefill {name}", n=300, seed=K)
+        del x, w, C
+        torch.cuda.empty_cache()
+
+
+def _expert_weights(hif4, experts, N, K, seed):
+    out = torch.empty(experts, N, K // 64, 36, dtype=torch.uint8, device="cuda")
+    step = 16                                          # BF16 sources are drawn 16 experts at a time
+    for e0 in range(0, experts, step):
+        w = wl.gaussian(step * N, K, 0.02, seed=seed + e0, device="cuda")
+        hif4.hif4_quantize(w, out=out[e0:e0 + step].view(step * N, K // 64, 36))
+        del w
+    return out
+
+
+def test_moe_layer_grouped_full_size(hif4):
+    """Config 5: 4096 tokens, top-8 of 256 experts under Zipf(1.1) popularity, both expert linears."""
+    r = wl.moe_routing(device="cuda")
+    off = r["offsets"]
+    counts = r["counts"].cpu().numpy()
+    total = int(off[-1])
+    assert total == wl.MOE_TOKENS * wl.MOE_TOPK and len(counts) == wl.MOE_EXPERTS
+    off_h = off.cpu().numpy()
+    order = np.argsort(counts)
+    picks = [int(order[-1]), int(order[0]), int(order[len(order) // 2]), int(order[-2]), int(order[len(order) // 4])]
+    for (K, N, seed) in ((wl.MOE_HIDDEN, 2 * wl.MOE_INTER, 5100), (wl.MOE_INTER, wl.MOE_HIDDEN, 5200)):
+        a = hif4.hif4_quantize(wl.outlier_channel_activations(total, K, seed=seed, device="cuda"))
+        b = _expert_weights(hif4, wl.MOE_EXPERTS, N, K, seed + 1)
+        C = hif4.hif4_grouped_gemm(a, b, off)
+        for g in picks:
+            lo, hi = int(off_h[g]), int(off_h[g + 1])
+            if hi > lo:
+                _sampled_entries(hif4, a[lo:hi], b[g], C[lo:hi], f"moe K={K} expert {g} ({hi - lo} rows)", n=60, seed=g)
+        del a, b, C
+        torch.cuda.empty_cache()
