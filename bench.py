@@ -35,7 +35,8 @@ SHAPES = [(M, K, N, name) for M in wl.LLAMA3_8B_M for (name, K, N) in wl.LLAMA3_
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (None until a capture exists for that kernel).
-NCU_DRAM_BYTES_PER_LAUNCH = {"gemm_tc2_kernel": None, "quantize_bf16_kernel@2^28": None}
+NCU_DRAM_BYTES_PER_LAUNCH = {"gemm_tc2_kernel": 265.4e6,      # captured on M=4096 N=14336 K=4096 (algorithmic 277.3e6)
+                             "quantize_bf16_kernel@2^28": 659.3e6}
 
 
 def load_peaks():
@@ -217,7 +218,8 @@ def run_cuda(args):
                 "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                 "frac": round(achieved / peaks["bf16_tflops_sustained"], 4),
                 "frac_of_burst_peak": round(achieved / peaks["bf16_tflops"], 4), "peak_kind": f"of {peak_kind} (sustained)",
-                "traffic": NCU_DRAM_BYTES_PER_LAUNCH["gemm_tc2_kernel"]}
+                "traffic": NCU_DRAM_BYTES_PER_LAUNCH["gemm_tc2_kernel"],
+                "traffic_note": "dram bytes of the M=4096 N=14336 K=4096 launch (profiles/gemm_tc2_kernel_4096x14336x4096.md)"}
 
     out = {
         "metric": METRIC, "value": round(value, 2), "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
@@ -232,6 +234,7 @@ def run_cuda(args):
 
     if rank == 0 and world == 1:
         out["roofline_quantize"] = measure_quantize_roofline(hif4, dev, peaks, peak_kind)
+        out["reference_points"] = measure_reference_points(dev)
     out["e2e"] = measure_e2e(hif4, dev, weights, world, args)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
@@ -265,6 +268,41 @@ def measure_quantize_roofline(hif4, dev, peaks, peak_kind):
             "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(gbs / peaks["hbm_gbs"], 4),
             "peak_kind": f"of {peak_kind}", "frac_of_nominal_8tbs": round(gbs / 8000.0, 4),
             "traffic": NCU_DRAM_BYTES_PER_LAUNCH["quantize_bf16_kernel@2^28"], "us_per_launch": round(ms * 1e3, 1)}
+
+
+def measure_reference_points(dev):
+    """Context only: the same (M, N, K) through the box's library GEMMs -- native NVFP4 block-scaled
+    (torch._scaled_mm on packed FP4 with one E4M3 scale per 16 values, random bits: time only) and BF16
+    (torch.matmul).  Neither is part of the HiF4 path."""
+    M, N, K = 4096, 14336, 4096
+    out = {"shape": [M, N, K]}
+
+    def timed(fn):
+        fn(); torch.cuda.synchronize()
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        for _ in range(20):
+            fn()
+        e.record(); torch.cuda.synchronize()
+        us = s.elapsed_time(e) / 20 * 1e3
+        return {"us": round(us, 1), "tflops": round(flops(M, K, N) / us / 1e6, 1)}
+
+    try:
+        a = torch.randint(0, 255, (M, K // 2), dtype=torch.uint8, device=dev).view(torch.float4_e2m1fn_x2)
+        b = torch.randint(0, 255, (N, K // 2), dtype=torch.uint8, device=dev).view(torch.float4_e2m1fn_x2)
+        cols = (K // 16 + 3) // 4 * 4
+        sa = torch.ones(((M + 127) // 128 * 128) * cols, device=dev).to(torch.float8_e4m3fn)
+        sb = torch.ones(((N + 127) // 128 * 128) * cols, device=dev).to(torch.float8_e4m3fn)
+        out["nvfp4_scaled_mm"] = timed(lambda: torch._scaled_mm(a, b.t(), sa, sb, out_dtype=torch.bfloat16))
+    except Exception as ex:                                   # noqa: BLE001 - any failure means "not on this box"
+        out["nvfp4_scaled_mm"] = {"unavailable": f"{type(ex).__name__}: {str(ex)[:120]}"}
+    try:
+        a = torch.randn(M, K, device=dev, dtype=torch.bfloat16)
+        b = torch.randn(N, K, device=dev, dtype=torch.bfloat16)
+        out["bf16_matmul"] = timed(lambda: torch.matmul(a, b.t()))
+    except Exception as ex:                                   # noqa: BLE001
+        out["bf16_matmul"] = {"unavailable": f"{type(ex).__name__}: {str(ex)[:120]}"}
+    return out
 
 
 def measure_e2e(hif4, dev, weights, world, args):
@@ -411,7 +449,10 @@ def run_case(spec: str):
         r = wl.moe_routing(tokens=tokens, experts=experts, topk=min(8, experts), device=dev)
         total = int(r["offsets"][-1])
         a = hif4.hif4_quantize(wl.outlier_channel_activations(total, K, seed=3, device=dev))
-        b = hif4.hif4_quantize(wl.gaussian(experts * N, K, 0.02, seed=4, device=dev)).view(experts, N, K // 64, 36)
+        b = torch.empty(experts, N, K // 64, 36, dtype=torch.uint8, device=dev)
+        for e0 in range(0, experts, 16):                    # BF16 sources are drawn 16 experts at a time
+            n_e = min(16, experts - e0)
+            hif4.hif4_quantize(wl.gaussian(n_e * N, K, 0.02, seed=4 + e0, device=dev), out=b[e0:e0 + n_e].view(n_e * N, K // 64, 36))
         c = torch.empty(total, N, dtype=torch.float32, device=dev)
         ws = torch.empty(max(hif4.hif4_grouped_gemm_workspace(experts, total, N, K), 1), dtype=torch.uint8, device=dev)
         fn = lambda: hif4.hif4_grouped_gemm(a, b, r["offsets"], out=c, workspace=ws)
