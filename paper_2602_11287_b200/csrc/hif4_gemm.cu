@@ -87,6 +87,13 @@ extern "C" hif4_status hif4_grouped_gemm(const void* A_units, const void* B_unit
   }
   const bool tc_ok = g_gemm_path != 1 &&
                      gemm_tc_supported(A_units, B_units, total_rows, static_cast<int64_t>(num_groups) * N, N, K);
+  if (tc_ok && g_gemm_path != 2 && N < (1ll << 31) - 256 && static_cast<int64_t>(num_groups) * N < (1ll << 31) - 256) {
+    // CTA pairs, swapped operands: padding of small experts costs 32 rows instead of 128
+    if (!workspace || workspace_bytes < grouped_tc2_workspace_bytes(num_groups, total_rows)) return HIF4_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return HIF4_ERR_ALIGN;
+    return launch_grouped_gemm_tc2(A_units, B_units, C, group_offsets_dev, num_groups, total_rows, N, K, ldc,
+                                   workspace, st);
+  }
   if (tc_ok) {
     const size_t need = grouped_tc_workspace_bytes(num_groups, total_rows);
     if (!workspace || workspace_bytes < need) return HIF4_ERR_WORKSPACE;

@@ -1,0 +1,339 @@
+// Grouped (MoE) tensor-core HiF4 GEMM on CTA pairs with the operands swapped: per expert g,
+// C[off[g]:off[g+1], :] = A[off[g]:off[g+1], :] * B[g]^T (Eq. 3 summed over unit pairs).
+//
+// Experts get very different numbers of rows (a few hot ones thousands, the median a few dozen), so
+// the tokens go on the flexible side of the MMA: a work unit is 256 weight rows of one expert (the
+// MMA's M side, 128 rows per CTA of the pair) times a token tile of T rows of that expert, T a multiple
+// of 32 up to 256 (the MMA's N side, T/2 rows per CTA).  A unit decodes 128 weight rows + T/2 token rows
+// per CTA and 64-wide K block, so a 40-row expert costs little more than the decode of its weights,
+// which every row of the expert needs anyway.  The accumulator holds C transposed (lane = weight row,
+// column = token); the epilogue stores it back with 32 lanes writing 32 consecutive columns of one
+// token's row, which is coalesced without staging and lets the last tile of a group stop at its end.
+//
+// Pipeline, barriers and bounded waits are those of the dense CTA-pair kernel: TMA producer warp (raw
+// units, K = 256 per stage, each CTA fetches its own rows), 16 decode warps, the MMA-issuing thread
+// on rank 0 with multicast commits, 4 epilogue warps, two accumulator stages.
+#include "hif4_common.cuh"
+#include "hif4_gemm_internal.cuh"
+#include "hif4_tc2_common.cuh"
+
+namespace hif4 {
+namespace {
+
+constexpr int kWRows = 128;                           // weight rows per CTA (256 per pair)
+constexpr int kMaxTok = 256;                          // token rows per unit (128 per CTA)
+constexpr int kRawHalfBytes = 128 * kRawRowBytes;     // 18432
+constexpr int kRawStageBytes = 2 * kRawHalfBytes;     // weight rows then token rows
+constexpr int kDecHalfBytes = 128 * 128;              // 128 rows x 64 BF16
+constexpr int kDecStageBytes = 2 * kDecHalfBytes;
+constexpr int kRawStages = 2;
+constexpr int kDecStages = 4;
+constexpr int kTmemCols = 512;
+
+constexpr int kDecodeWarp0 = 6;
+constexpr int kDecodeThreads = 512;
+constexpr int kThreads = kDecodeWarp0 * 32 + kDecodeThreads;   // 704
+constexpr int kSmemBytes = 1024 + kDecStages * kDecStageBytes + kRawStages * kRawStageBytes + 256 + 1024;
+
+// tcgen05.mma kind::f16 descriptor without the N field: D = F32, A = B = BF16, K-major, M = 256.
+constexpr uint32_t kInstrDescM256 = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(256 >> 4) << 24);
+
+struct TokTile { int tok0; int tok_end; int group; int T; };     // T = rows of the tile rounded up to 32
+
+struct GroupedParams {
+  float* C;
+  int64_t ldc;
+  int64_t N;            // weight rows per expert = columns of C
+  int num_kc;           // K / 256
+  int n_wtiles;         // ceil(N / 256)
+  int max_entries;
+  const TokTile* table;
+  unsigned int* error_word;
+  DecodeMul mul;
+};
+
+// One thread walks the offsets: every group is cut into token tiles of 256 rows, the last one padded
+// to a multiple of 32; unused entries are marked invalid.
+__global__ void build_toktile_table_kernel(const int64_t* __restrict__ offsets, int num_groups, TokTile* table,
+                                           int max_entries) {
+  __shared__ int s_total;
+  if (threadIdx.x == 0) {
+    int n = 0;
+    for (int g = 0; g < num_groups; ++g) {
+      const int64_t lo = offsets[g], hi = offsets[g + 1];
+      for (int64_t r = lo; r < hi && n < max_entries; r += kMaxTok) {
+        const int rows = static_cast<int>(hi - r < kMaxTok ? hi - r : kMaxTok);
+        table[n].tok0 = static_cast<int>(r);
+        table[n].tok_end = static_cast<int>(hi);
+        table[n].group = g;
+        table[n].T = (rows + 31) & ~31;
+        ++n;
+      }
+    }
+    s_total = n;
+  }
+  __syncthreads();
+  for (int i = s_total + threadIdx.x; i < max_entries; i += blockDim.x) {
+    table[i].tok0 = 0; table[i].tok_end = 0; table[i].group = -1; table[i].T = 0;
+  }
+}
+
+struct Unit { int tok0; int tok_end; int T; int w_row0; int n0; bool valid; };
+__device__ __forceinline__ Unit unit_of(const GroupedParams& p, int u) {
+  const int e = u / p.n_wtiles, wt = u - e * p.n_wtiles;
+  const TokTile t = p.table[e];
+  Unit r;
+  r.valid = t.group >= 0;
+  r.tok0 = t.tok0; r.tok_end = t.tok_end; r.T = t.T;
+  r.n0 = wt * 256;
+  r.w_row0 = static_cast<int>(t.group * p.N) + r.n0;
+  return r;
+}
+
+// Decodes the two units held in raw words L[kOff..] into decoded stages 2h and 2h+1 (skipped for rows
+// that the tile does not use; the barrier protocol runs either way).
+template <int kOff>
+__device__ __forceinline__ bool decode_two_units_g(const uint32_t (&L)[20], bool active, const uint32_t (&chunk_addr)[8],
+                                                   uint32_t lut, const DecodeMul& mul, uint32_t dec_empty0,
+                                                   uint32_t dec_full0_leader, uint32_t parity_free,
+                                                   volatile uint32_t* abort_flag) {
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    if (!__all_sync(0xFFFFFFFFu, mbar_wait(dec_empty0 + 8 * u, parity_free, abort_flag))) return false;
+    if (active) decode_unit_balanced(L[kOff + 9 * u], &L[kOff + 9 * u + 1], chunk_addr, u * kDecStageBytes, lut, mul);
+    fence_proxy_async_smem();
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive_cluster(dec_full0_leader + 8 * u);
+  }
+  return true;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constant__ CUtensorMap tmW,
+                 const GroupedParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t dec_base = smem_base;                                        // 1024-byte aligned stages
+  const uint32_t raw_base = dec_base + kDecStages * kDecStageBytes;
+  const uint32_t bar_base = raw_base + kRawStages * kRawStageBytes;
+  const uint32_t raw_full = bar_base, raw_empty = bar_base + 16, dec_full = bar_base + 32, dec_empty = bar_base + 64,
+                 tmem_full = bar_base + 96, tmem_empty = bar_base + 112;
+  uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(gen_base + (bar_base - smem_base) + 128);
+  volatile uint32_t* abort_flag = tmem_ptr_smem + 1;
+  const uint32_t lut = bar_base + 256;
+  if (threadIdx.x < 256)
+    reinterpret_cast<uint32_t*>(gen_base + (lut - smem_base))[threadIdx.x] = spread_e8_entry(threadIdx.x);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+  const int total_units = p.max_entries * p.n_wtiles;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kRawStages; ++s) {
+      mbar_init(raw_full + 8 * s, 1);
+      mbar_init(raw_empty + 8 * s, kDecodeThreads);
+    }
+    for (int s = 0; s < kDecStages; ++s) {
+      mbar_init(dec_full + 8 * s, kDecodeThreads / 32);   // 8 warps of each CTA per stage (used on rank 0)
+      mbar_init(dec_empty + 8 * s, 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(tmem_full + 8 * s, 1);
+      mbar_init(tmem_empty + 8 * s, 8);                   // 4 epilogue warps of each CTA (used on rank 0)
+    }
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bar_base + 128),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();            // the peer's barriers are initialised before anyone arrives on them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_ptr_smem;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      uint32_t n = 0;
+      bool ok = true;
+      for (int u = pair; u < total_units && ok; u += num_pairs) {
+        const Unit un = unit_of(p, u);
+        if (!un.valid) continue;
+        for (int kc = 0; kc < p.num_kc; ++kc, ++n) {
+          const uint32_t s = n & 1u, ph = (n >> 1) & 1u;
+          if (!(ok = mbar_wait(raw_empty + 8 * s, ph ^ 1u, abort_flag, 128))) break;
+          mbar_expect_tx(raw_full + 8 * s, kRawStageBytes);
+          const uint32_t dst = raw_base + s * kRawStageBytes;
+          tma_load_2d(dst, &tmW, kc * kRawRowBytes, un.w_row0 + static_cast<int>(rank) * kWRows, raw_full + 8 * s);
+          tma_load_2d(dst + kRawHalfBytes, &tmTok, kc * kRawRowBytes, un.tok0 + static_cast<int>(rank) * (un.T >> 1),
+                      raw_full + 8 * s);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer (rank 0 only)
+    if (rank == 0 && lane == 0) {
+      uint32_t n = 0, ucount = 0;
+      bool ok = true;
+      for (int u = pair; u < total_units && ok; u += num_pairs) {
+        const Unit un = unit_of(p, u);
+        if (!un.valid) continue;
+        const uint32_t acc = ucount & 1u, aph = (ucount >> 1) & 1u;
+        if (!(ok = mbar_wait_cluster(tmem_empty + 8 * acc, aph ^ 1u, abort_flag))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * kMaxTok;
+        const uint32_t idesc = kInstrDescM256 | (static_cast<uint32_t>(un.T >> 3) << 17);
+        for (int kc = 0; kc < p.num_kc && ok; ++kc, ++n) {
+          // stages 0 and 2 are filled first (see the dense pair kernel): consume 0, 2, 1, 3
+#pragma unroll
+          for (int i = 0; i < kDecStages; ++i) {
+            const int st = ((i & 1) << 1) | (i >> 1);
+            if (!(ok = mbar_wait_cluster(dec_full + 8 * st, n & 1u, abort_flag))) break;
+            tc_fence_after();
+            const uint64_t adesc = make_desc(dec_base + st * kDecStageBytes);                  // weights: M side
+            const uint64_t bdesc = make_desc(dec_base + st * kDecStageBytes + kDecHalfBytes);  // tokens: N side
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              tc2_mma(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kc | i | kk) != 0 ? 1u : 0u);
+            tc2_commit_both(dec_empty + 8 * st);
+          }
+        }
+        if (!ok) break;
+        tc2_commit_both(tmem_full + 8 * acc);
+        ++ucount;
+      }
+    }
+  } else if (warp < kDecodeWarp0) {
+    // ---------------------------------------------------------------- epilogue: C^T tile -> rows of C
+    const int q = warp & 3;                      // TMEM lane quadrant this warp may read
+    const uint32_t tmem_empty_leader = mapa(tmem_empty, 0);
+    uint32_t ucount = 0;
+    for (int u = pair; u < total_units; u += num_pairs) {
+      const Unit un = unit_of(p, u);
+      if (!un.valid) continue;
+      const uint32_t acc = ucount & 1u, aph = (ucount >> 1) & 1u;
+      if (!__all_sync(0xFFFFFFFFu, mbar_wait(tmem_full + 8 * acc, aph, abort_flag, 256))) break;
+      tc_fence_after();
+      const int64_t col = static_cast<int64_t>(un.n0) + rank * kWRows + q * 32 + lane;      // column of C = weight row
+      const bool col_ok = col < p.N;
+      const int chunks = un.T >> 4;
+#pragma unroll 1
+      for (int c = 0; c < chunks; ++c) {
+        uint32_t r[16];
+        tc_ld16(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kMaxTok + c * 16, r);
+        tc_wait_ld();
+        if (c == chunks - 1) {                   // accumulator fully read: hand it back before the stores
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + 8 * acc);
+        }
+        const int tok = un.tok0 + c * 16;
+        float* cp = p.C + static_cast<int64_t>(tok) * p.ldc + col;
+#pragma unroll
+        for (int v = 0; v < 16; ++v)
+          if (col_ok && tok + v < un.tok_end) cp[static_cast<int64_t>(v) * p.ldc] = __uint_as_float(r[v]);
+      }
+      ++ucount;
+    }
+  } else {
+    // ---------------------------------------------------------------- decode
+    const int d = threadIdx.x - kDecodeWarp0 * 32;            // 0..511
+    const int h = d >> 8;                                     // which unit pair of the raw chunk
+    const int row = d & 255;                                  // 0..127 weight rows, 128..255 token rows
+    const uint32_t r7 = static_cast<uint32_t>(row) & 7u;
+    const uint32_t raw_row = static_cast<uint32_t>(row) * kRawRowBytes + static_cast<uint32_t>(h) * 64u;
+    const uint32_t dec_row = dec_base + static_cast<uint32_t>(2 * h) * kDecStageBytes + static_cast<uint32_t>(row) * 128u;
+    uint32_t chunk_addr[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) chunk_addr[j] = dec_row + ((static_cast<uint32_t>(j) ^ r7) << 4);
+    const uint32_t dec_empty0 = dec_empty + 16 * h;
+    const uint32_t dec_full0_leader = mapa(dec_full, 0) + 16 * h;
+    uint32_t n = 0;
+    bool ok = true;
+    for (int u = pair; u < total_units && ok; u += num_pairs) {
+      const Unit un = unit_of(p, u);
+      if (!un.valid) continue;
+      const bool active = row < 128 || (row - 128) < (un.T >> 1);
+      for (int kc = 0; kc < p.num_kc && ok; ++kc, ++n) {
+        const uint32_t s = n & 1u, ph = (n >> 1) & 1u;
+        if (!(ok = __all_sync(0xFFFFFFFFu, mbar_wait(raw_full + 8 * s, ph, abort_flag)))) break;
+        uint32_t L[20];
+        const uint32_t src = raw_base + s * kRawStageBytes + raw_row;
+#pragma unroll
+        for (int i = 0; i < 5; ++i) {
+          const uint4 v = lds128(src + 16 * i);
+          L[4 * i] = v.x; L[4 * i + 1] = v.y; L[4 * i + 2] = v.z; L[4 * i + 3] = v.w;
+        }
+        fence_proxy_async_smem();                // reads ordered before the async proxy refills the stage
+        mbar_arrive(raw_empty + 8 * s);
+        if (h == 0) ok = decode_two_units_g<0>(L, active, chunk_addr, lut, p.mul, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
+        else ok = decode_two_units_g<2>(L, active, chunk_addr, lut, p.mul, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncwarp();
+  if (*abort_flag) {
+    const uint64_t t0 = global_ns();
+    while (global_ns() - t0 < 2000000ull) {}     // let copies and MMAs that are still in flight land
+    if (threadIdx.x == 0) atomicExch(p.error_word, 1u);
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();            // neither CTA leaves while the other may still read its shared memory or arrive on its barriers
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+}  // namespace
+
+size_t grouped_tc2_workspace_bytes(int num_groups, int64_t total_rows) {
+  const int64_t max_entries = ceil_div64(total_rows, kMaxTok) + num_groups;
+  return static_cast<size_t>((max_entries * static_cast<int64_t>(sizeof(TokTile)) + 255) / 256 * 256);
+}
+
+hif4_status launch_grouped_gemm_tc2(const void* A, const void* B, float* C, const int64_t* offsets, int num_groups,
+                                    int64_t total_rows, int64_t N, int64_t K, int64_t ldc, void* workspace,
+                                    cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gemm_tc2g_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+      return HIF4_ERR_CUDA;
+    attr_set = true;
+  }
+  const int max_entries = static_cast<int>(ceil_div64(total_rows, kMaxTok) + num_groups);
+  TokTile* table = static_cast<TokTile*>(workspace);
+  build_toktile_table_kernel<<<1, 256, 0, st>>>(offsets, num_groups, table, max_entries);
+  note_launch();
+  if (cudaGetLastError() != cudaSuccess) return HIF4_ERR_CUDA;
+  CUtensorMap tmTok, tmW;
+  const int64_t upr = K / kUnitElems;
+  if (!make_unit_map(&tmTok, A, total_rows, upr, 128) || !make_unit_map(&tmW, B, static_cast<int64_t>(num_groups) * N, upr, kWRows))
+    return HIF4_ERR_CUDA;
+  GroupedParams p{};
+  p.C = C; p.ldc = ldc; p.N = N;
+  p.num_kc = static_cast<int>(K / (kRawUnits * kUnitElems));
+  p.n_wtiles = static_cast<int>(ceil_div64(N, 256));
+  p.max_entries = max_entries;
+  p.table = table;
+  p.error_word = device_error_word();
+  if (!p.error_word) return HIF4_ERR_CUDA;
+  p.mul = make_decode_mul();
+  const int64_t units = static_cast<int64_t>(max_entries) * p.n_wtiles;
+  if (units > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
+  const int pairs = static_cast<int>(units < sm_count() / 2 ? units : sm_count() / 2);
+  gemm_tc2g_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tmTok, tmW, p);
+  note_launch();
+  return launch_status();
+}
+
+}  // namespace hif4

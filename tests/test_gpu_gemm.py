@@ -203,10 +203,13 @@ def test_tensor_core_kernel_c_rows_not_16_byte_aligned(tc_path):
 
 
 def test_tensor_core_grouped(tc_path):
+    """Path 2 = single-CTA kernel with 128-row tiles, path 3 = CTA pairs with swapped operands."""
     hif4 = tc_path
     _grouped_case(hif4, [3, 0, 70, 1, 0, 129, 64, 0, 300], N=300, K=256, seed=61)
     _grouped_case(hif4, [0, 0, 5], N=64, K=512, seed=62)
     _grouped_case(hif4, [513], N=256, K=256, seed=63)
+    _grouped_case(hif4, [31, 32, 33, 255, 256, 257, 0, 16, 700], N=520, K=768, seed=64)
+    _grouped_case(hif4, [1] * 40, N=257, K=256, seed=65)
 
 
 def test_tensor_core_prefill_shape_sampled(tc_path):
