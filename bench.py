@@ -482,11 +482,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--gemm-path", type=int, default=0, help="with --case: kernel selection, see hif4_set_gemm_path")
     ap.add_argument("--case", default=None,
                     help="run one kernel a few times instead of the benchmark (for ncu captures): "
                          "gemm:M,N,K | quantize:LOG2_ELEMS | dequantize:LOG2_ELEMS | grouped:TOKENS,EXPERTS,N,K")
     args = ap.parse_args()
     if args.case:
+        if args.gemm_path:
+            import paper_2602_11287_b200 as hif4
+            hif4.hif4_set_gemm_path(args.gemm_path)
         run_case(args.case)
         return
     if args.impl == "reference":

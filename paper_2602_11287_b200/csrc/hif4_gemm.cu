@@ -56,6 +56,9 @@ extern "C" hif4_status hif4_gemm(const void* A_units, const void* B_units, float
   const bool tc_ok = g_gemm_path != 1 && gemm_tc_supported(A_units, B_units, M, N, N, K);
   if (tc_ok && g_gemm_path != 2 && (g_gemm_path == 3 || M >= kPairMinM) && gemm_tc2_supported(A_units, B_units, M, N, K))
     return launch_gemm_tc2(A_units, B_units, C, M, N, K, ldc, st);
+  // few rows: the pair kernel with the operands swapped pads them to 32 instead of 128
+  if (tc_ok && g_gemm_path == 0 && M > kGemvMaxM && M < kPairMinM && gemm_tc2_supported(A_units, B_units, M, N, K))
+    return launch_gemm_tc2_swapped(A_units, B_units, C, M, N, K, ldc, st);
   if (tc_ok && (g_gemm_path >= 2 || M > kGemvMaxM)) return launch_gemm_tc(A_units, B_units, C, M, N, K, ldc, st);
   return launch_gemm_simt(A_units, B_units, C, M, N, K, ldc, st);
 }

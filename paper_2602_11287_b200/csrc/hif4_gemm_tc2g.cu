@@ -47,7 +47,8 @@ struct GroupedParams {
   int num_kc;           // K / 256
   int n_wtiles;         // ceil(N / 256)
   int max_entries;
-  const TokTile* table;
+  const TokTile* table;     // nullptr: one dense problem of dense_rows token rows (a single tile)
+  int dense_rows;
   unsigned int* error_word;
   DecodeMul mul;
 };
@@ -81,7 +82,7 @@ __global__ void build_toktile_table_kernel(const int64_t* __restrict__ offsets, 
 struct Unit { int tok0; int tok_end; int T; int w_row0; int n0; bool valid; };
 __device__ __forceinline__ Unit unit_of(const GroupedParams& p, int u) {
   const int e = u / p.n_wtiles, wt = u - e * p.n_wtiles;
-  const TokTile t = p.table[e];
+  const TokTile t = p.table ? p.table[e] : TokTile{0, p.dense_rows, 0, (p.dense_rows + 31) & ~31};
   Unit r;
   r.valid = t.group >= 0;
   r.tok0 = t.tok0; r.tok_end = t.tok_end; r.T = t.T;
@@ -294,7 +295,42 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
   }
 }
 
+hif4_status launch_swapped(const void* A, const void* B, int64_t a_rows, int64_t b_rows, GroupedParams p, int64_t K,
+                           cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gemm_tc2g_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+      return HIF4_ERR_CUDA;
+    attr_set = true;
+  }
+  CUtensorMap tmTok, tmW;
+  const int64_t upr = K / kUnitElems;
+  if (!make_unit_map(&tmTok, A, a_rows, upr, 128) || !make_unit_map(&tmW, B, b_rows, upr, kWRows)) return HIF4_ERR_CUDA;
+  p.num_kc = static_cast<int>(K / (kRawUnits * kUnitElems));
+  p.n_wtiles = static_cast<int>(ceil_div64(p.N, 256));
+  p.error_word = device_error_word();
+  if (!p.error_word) return HIF4_ERR_CUDA;
+  p.mul = make_decode_mul();
+  const int64_t units = static_cast<int64_t>(p.max_entries) * p.n_wtiles;
+  if (units > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
+  const int pairs = static_cast<int>(units < sm_count() / 2 ? units : sm_count() / 2);
+  gemm_tc2g_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tmTok, tmW, p);
+  note_launch();
+  return launch_status();
+}
+
 }  // namespace
+
+// Dense problem with few rows (M <= 128): the same kernel with a single token tile.
+hif4_status launch_gemm_tc2_swapped(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K,
+                                    int64_t ldc, cudaStream_t st) {
+  GroupedParams p{};
+  p.C = C; p.ldc = ldc; p.N = N;
+  p.max_entries = 1;
+  p.table = nullptr;
+  p.dense_rows = static_cast<int>(M);
+  return launch_swapped(A, B, M, N, p, K, st);
+}
 
 size_t grouped_tc2_workspace_bytes(int num_groups, int64_t total_rows) {
   const int64_t max_entries = ceil_div64(total_rows, kMaxTok) + num_groups;
@@ -304,36 +340,16 @@ size_t grouped_tc2_workspace_bytes(int num_groups, int64_t total_rows) {
 hif4_status launch_grouped_gemm_tc2(const void* A, const void* B, float* C, const int64_t* offsets, int num_groups,
                                     int64_t total_rows, int64_t N, int64_t K, int64_t ldc, void* workspace,
                                     cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_tc2g_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-      return HIF4_ERR_CUDA;
-    attr_set = true;
-  }
   const int max_entries = static_cast<int>(ceil_div64(total_rows, kMaxTok) + num_groups);
   TokTile* table = static_cast<TokTile*>(workspace);
   build_toktile_table_kernel<<<1, 256, 0, st>>>(offsets, num_groups, table, max_entries);
   note_launch();
   if (cudaGetLastError() != cudaSuccess) return HIF4_ERR_CUDA;
-  CUtensorMap tmTok, tmW;
-  const int64_t upr = K / kUnitElems;
-  if (!make_unit_map(&tmTok, A, total_rows, upr, 128) || !make_unit_map(&tmW, B, static_cast<int64_t>(num_groups) * N, upr, kWRows))
-    return HIF4_ERR_CUDA;
   GroupedParams p{};
   p.C = C; p.ldc = ldc; p.N = N;
-  p.num_kc = static_cast<int>(K / (kRawUnits * kUnitElems));
-  p.n_wtiles = static_cast<int>(ceil_div64(N, 256));
   p.max_entries = max_entries;
   p.table = table;
-  p.error_word = device_error_word();
-  if (!p.error_word) return HIF4_ERR_CUDA;
-  p.mul = make_decode_mul();
-  const int64_t units = static_cast<int64_t>(max_entries) * p.n_wtiles;
-  if (units > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
-  const int pairs = static_cast<int>(units < sm_count() / 2 ? units : sm_count() / 2);
-  gemm_tc2g_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tmTok, tmW, p);
-  note_launch();
-  return launch_status();
+  return launch_swapped(A, B, total_rows, static_cast<int64_t>(num_groups) * N, p, K, st);
 }
 
 }  // namespace hif4

@@ -56,6 +56,21 @@ def test_small_and_ragged_shapes(hif4, M, N, K):
     check_full(hif4, hif4.hif4_quantize(a), hif4.hif4_quantize(b), f"{M}x{N}x{K}")
 
 
+@pytest.mark.parametrize("M,N,K", [(17, 300, 256), (40, 257, 768), (100, 1000, 1024), (128, 512, 2048), (65, 31, 256)])
+def test_few_rows_default_path(hif4, M, N, K):
+    """17 <= M <= 128 with K % 256 == 0 goes to the CTA-pair kernel with swapped operands."""
+    g = torch.Generator(device="cuda"); g.manual_seed(M * 13 + N)
+    a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
+    b = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
+    out = torch.full((M + 2, N + 5), -5.0, dtype=torch.float32, device="cuda")
+    before = hif4.launch_count()
+    C = check_full(hif4, a, b, f"few rows {M}x{N}x{K}", out=out[1:M + 1, 2:N + 2])
+    assert hif4.launch_count() - before == 1
+    assert (out[0] == -5.0).all() and (out[M + 1] == -5.0).all() and (out[:, :2] == -5.0).all() and (out[:, N + 2:] == -5.0).all()
+    assert torch.equal(C.contiguous(), hif4.hif4_gemm(a, b)), "two runs differ"
+    assert hif4.hif4_last_device_status() == 0
+
+
 def test_random_units_all_scales_and_strided_c(hif4):
     rng = np.random.default_rng(21)
     M, N, upr = 70, 90, 4
