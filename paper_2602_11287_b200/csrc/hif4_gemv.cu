@@ -8,12 +8,12 @@
 //   2. gemv_kernel: one CTA owns 16 * kRowGroups weight rows and the whole K range.  A producer warp
 //      streams, per K = 256 chunk, the CTA's packed weight rows (one 2-D TMA box, 144 bytes per row) and
 //      the tokens' chunk (one bulk copy, L2-resident) through an 8-stage ring.  Consumer warp (rg, ks)
-//      owns 16 weight rows and unit ks of every chunk (four K slices per row group, so that even a
-//      narrow problem has enough warps in flight): lane (g, q) reads the metadata word and code words
+//      owns 16 weight rows and unit ks of every kChunkWays-th chunk (8 or 16 K slices per row group, so
+//      that even a narrow problem has enough warps in flight to hide the decode latency): lane (g, q) reads the metadata word and code words
 //      2q, 2q+1 of rows g and g+8, decodes them in registers straight into the A fragments (weights are
 //      the 16-row MMA operand), reads the matching token fragments from shared memory and issues four
 //      BF16 MMAs with FP32 accumulators.  Inside a unit the K order is permuted the same way on both
-//      operands.  The four K slices are summed through shared memory in a fixed order.
+//      operands.  The K slices are summed through shared memory in a fixed order.
 // Results are deterministic (no atomics).  Every mbarrier wait is bounded.
 #include "hif4_common.cuh"
 #include "hif4_gemm_internal.cuh"
@@ -106,10 +106,10 @@ gemv_prepare_tokens_kernel(const uint32_t* __restrict__ A, int M, int m_pad, int
   }
 }
 
-template <int kRowGroups, int kTokTiles>
-__global__ void __launch_bounds__((4 * kRowGroups + 1) * 32)
+template <int kRowGroups, int kTokTiles, int kChunkWays>
+__global__ void __launch_bounds__((4 * kChunkWays * kRowGroups + 1) * 32)
 gemv_kernel(const __grid_constant__ CUtensorMap tmB, const GemvParams p) {
-  constexpr int kWarps = 4 * kRowGroups;                           // consumer warps
+  constexpr int kWarps = 4 * kChunkWays * kRowGroups;              // consumer warps
   constexpr int kRows = 16 * kRowGroups;
   constexpr int kWeightBytes = kRows * kRawRowBytes;
   constexpr int kTokBytes = 8 * kTokTiles * kTokChunkBytes;
@@ -129,7 +129,7 @@ gemv_kernel(const __grid_constant__ CUtensorMap tmB, const GemvParams p) {
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(full + 8 * s, 1);
-      mbar_init(empty + 8 * s, kWarps);
+      mbar_init(empty + 8 * s, 4 * kRowGroups);          // the warps that read one chunk
     }
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -151,13 +151,15 @@ gemv_kernel(const __grid_constant__ CUtensorMap tmB, const GemvParams p) {
     }
   } else {
     // ---------------------------------------------------------------- consumers: 16 weight rows x one K slice per warp
-    const int rg = warp % kRowGroups, ks = warp / kRowGroups;          // row group, unit of each chunk
+    // row group, K slice: unit (slice & 3) of the chunks kc = slice / 4 (mod kChunkWays)
+    const int rg = warp % kRowGroups, slice = warp / kRowGroups, ks = slice & 3, way = slice >> 2;
     const int g = lane >> 2, q = lane & 3;
-    float acc[kTokTiles][4];
+    // two accumulator sets per token tile, so that consecutive MMAs do not wait on one another
+    float acc[kTokTiles][4], acc2[kTokTiles][4];
 #pragma unroll
     for (int t = 0; t < kTokTiles; ++t)
 #pragma unroll
-      for (int i = 0; i < 4; ++i) acc[t][i] = 0.0f;
+      for (int i = 0; i < 4; ++i) acc[t][i] = acc2[t][i] = 0.0f;
     const uint32_t w_off0 = static_cast<uint32_t>(16 * rg + g) * kRawRowBytes + ks * kUnitBytes;   // MMA row g
     const uint32_t w_off1 = w_off0 + 8 * kRawRowBytes;                                               // MMA row g + 8
     // token g (and g + 8): words 2q and 2q+1 of unit ks, 16-byte groups swizzled by the token's parity
@@ -165,7 +167,7 @@ gemv_kernel(const __grid_constant__ CUtensorMap tmB, const GemvParams p) {
     const uint32_t t_lo = t_base + ((static_cast<uint32_t>(2 * q) ^ (g & 1u)) << 4);
     const uint32_t t_hi = t_base + ((static_cast<uint32_t>(2 * q + 1) ^ (g & 1u)) << 4);
     bool ok = true;
-    for (int kc = 0; kc < p.num_kc && ok; ++kc) {
+    for (int kc = way; kc < p.num_kc && ok; kc += kChunkWays) {
       const uint32_t s = kc % kStages, ph = (kc / kStages) & 1u;
       if (!(ok = __all_sync(0xFFFFFFFFu, mbar_wait(full + 8 * s, ph, abort_flag)))) break;
       const uint32_t st = smem_base + s * kStageBytes;
@@ -187,19 +189,23 @@ gemv_kernel(const __grid_constant__ CUtensorMap tmB, const GemvParams p) {
 #pragma unroll
       for (int t = 0; t < kTokTiles; ++t) {
         mma_bf16_16816(acc[t], a[0], b[0], a[1], b[1], x[t].x, x[t].y);
-        mma_bf16_16816(acc[t], a[2], b[2], a[3], b[3], x[t].z, x[t].w);
+        mma_bf16_16816(acc2[t], a[2], b[2], a[3], b[3], x[t].z, x[t].w);
         mma_bf16_16816(acc[t], a[4], b[4], a[5], b[5], y[t].x, y[t].y);
-        mma_bf16_16816(acc[t], a[6], b[6], a[7], b[7], y[t].z, y[t].w);
+        mma_bf16_16816(acc2[t], a[6], b[6], a[7], b[7], y[t].z, y[t].w);
       }
     }
-    // Sum the four K slices of every row group in a fixed order, then store.
+#pragma unroll
+    for (int t = 0; t < kTokTiles; ++t)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[t][i] += acc2[t][i];
+    // Sum the K slices of every row group in a fixed order, then store.
     float* mine = red + (static_cast<size_t>(warp) * 32 + lane) * (4 * kTokTiles);
 #pragma unroll
     for (int t = 0; t < kTokTiles; ++t)
 #pragma unroll
       for (int i = 0; i < 4; ++i) mine[4 * t + i] = acc[t][i];
-    asm volatile("bar.sync 1, %0;" ::"n"(kWarps * 32) : "memory");
-    if (ks == 0 && !*abort_flag) {
+    asm volatile("bar.sync 1, %0;" ::"n"(kWarps * 32) : "memory");     // consumer warps only
+    if (slice == 0 && !*abort_flag) {
       // acc[t]: {row g: tokens 2q, 2q+1; row g+8: tokens 2q, 2q+1} (+ 8 t)
       const int64_t n0 = row0 + 16 * rg + g;
 #pragma unroll
@@ -208,7 +214,7 @@ gemv_kernel(const __grid_constant__ CUtensorMap tmB, const GemvParams p) {
         for (int i = 0; i < 4; ++i) {
           float v = acc[t][i];
 #pragma unroll
-          for (int k = 1; k < 4; ++k)
+          for (int k = 1; k < 4 * kChunkWays; ++k)
             v += red[(static_cast<size_t>(k * kRowGroups + rg) * 32 + lane) * (4 * kTokTiles) + 4 * t + i];
           const int tok = 8 * t + 2 * q + (i & 1);
           const int64_t n = n0 + (i >> 1) * 8;
@@ -224,14 +230,14 @@ gemv_kernel(const __grid_constant__ CUtensorMap tmB, const GemvParams p) {
   }
 }
 
-template <int kRowGroups, int kTokTiles>
+template <int kRowGroups, int kTokTiles, int kChunkWays>
 hif4_status launch_gemv_t(const void* B, int64_t upr, const GemvParams& p, cudaStream_t st) {
   constexpr int kRows = 16 * kRowGroups;
   constexpr int smem = 128 + kStages * (kRows * kRawRowBytes + 8 * kTokTiles * kTokChunkBytes) +
-                       4 * kRowGroups * 32 * 4 * kTokTiles * 4 + 16 * kStages + 16;
+                       4 * kChunkWays * kRowGroups * 32 * 4 * kTokTiles * 4 + 16 * kStages + 16;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(gemv_kernel<kRowGroups, kTokTiles>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemv_kernel<kRowGroups, kTokTiles, kChunkWays>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return HIF4_ERR_CUDA;
     attr_set = true;
   }
@@ -239,7 +245,7 @@ hif4_status launch_gemv_t(const void* B, int64_t upr, const GemvParams& p, cudaS
   if (!make_unit_map(&tmB, B, p.N, upr, kRows)) return HIF4_ERR_CUDA;
   const int64_t blocks = ceil_div64(p.N, kRows);
   if (blocks > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
-  gemv_kernel<kRowGroups, kTokTiles><<<static_cast<unsigned>(blocks), (4 * kRowGroups + 1) * 32, smem, st>>>(tmB, p);
+  gemv_kernel<kRowGroups, kTokTiles, kChunkWays><<<static_cast<unsigned>(blocks), (4 * kChunkWays * kRowGroups + 1) * 32, smem, st>>>(tmB, p);
   note_launch();
   return launch_status();
 }
@@ -270,11 +276,11 @@ hif4_status launch_gemv(const void* A, const void* B, float* C, int64_t M, int64
   gemv_prepare_tokens_kernel<<<static_cast<unsigned>(ceil_div64(prep, 128)), 128, 0, st>>>(p.A, p.M, p.m_pad, upr, p.tokens);
   note_launch();
   if (cudaGetLastError() != cudaSuccess) return HIF4_ERR_CUDA;
-  // 16 weight rows (4 warps) per CTA for narrow problems, 32 rows (8 warps) once that still gives
-  // every SM two CTAs
+  // 16 weight rows per CTA with 16 K slices for narrow problems (few CTAs, so each needs many warps),
+  // 32 rows with 4 K slices per row group once that still gives every SM two CTAs
   const bool wide = N >= 64ll * sm_count();
-  if (p.m_pad == 8) return wide ? launch_gemv_t<2, 1>(B, upr, p, st) : launch_gemv_t<1, 1>(B, upr, p, st);
-  return wide ? launch_gemv_t<2, 2>(B, upr, p, st) : launch_gemv_t<1, 2>(B, upr, p, st);
+  if (p.m_pad == 8) return wide ? launch_gemv_t<2, 1, 1>(B, upr, p, st) : launch_gemv_t<1, 1, 4>(B, upr, p, st);
+  return wide ? launch_gemv_t<2, 2, 1>(B, upr, p, st) : launch_gemv_t<1, 2, 4>(B, upr, p, st);
 }
 
 }  // namespace hif4
