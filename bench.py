@@ -437,6 +437,13 @@ def run_case(spec: str):
         ws = torch.empty(max(hif4.hif4_gemm_workspace(M, N, K), 256), dtype=torch.uint8, device=dev)
         fn = lambda: hif4.hif4_gemm(a, b, out=c, workspace=ws)
         work = f"{flops(M, K, N) / 1e9:.1f} GFLOP, min traffic {gemm_min_bytes(M, K, N) / 1e6:.1f} MB"
+    elif kind in ("quantize32", "dequantize32"):
+        n = 2 ** nums[0]
+        x = wl.quantize_sweep(n, device=dev, dtype=torch.float32)
+        q = torch.empty(n // 4096, 64, 36, dtype=torch.uint8, device=dev)
+        hif4.hif4_quantize(x, out=q)
+        fn = (lambda: hif4.hif4_quantize(x, out=q)) if kind == "quantize32" else (lambda: hif4.hif4_dequantize(q, out=x))
+        work = f"{n * 4.5625 / 1e6:.1f} MB"
     elif kind in ("quantize", "dequantize"):
         n = 2 ** nums[0]
         x = wl.quantize_sweep(n, device=dev)
@@ -485,7 +492,8 @@ def main():
     ap.add_argument("--gemm-path", type=int, default=0, help="with --case: kernel selection, see hif4_set_gemm_path")
     ap.add_argument("--case", default=None,
                     help="run one kernel a few times instead of the benchmark (for ncu captures): "
-                         "gemm:M,N,K | quantize:LOG2_ELEMS | dequantize:LOG2_ELEMS | grouped:TOKENS,EXPERTS,N,K")
+                         "gemm:M,N,K | quantize:LOG2_ELEMS | dequantize:LOG2_ELEMS | quantize32 / dequantize32 (FP32 side) | "
+                         "grouped:TOKENS,EXPERTS,N,K")
     args = ap.parse_args()
     if args.case:
         if args.gemm_path:

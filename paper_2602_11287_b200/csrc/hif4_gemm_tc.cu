@@ -297,12 +297,8 @@ __global__ void build_mtile_table_kernel(const int64_t* __restrict__ offsets, in
 // ------------------------------------------------------------------------------------ host side
 hif4_status launch_tc(const void* A, const void* B, int64_t a_rows, int64_t b_rows, GemmParams p, int64_t K,
                       cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-      return HIF4_ERR_CUDA;
-    attr_set = true;
-  }
+  static uint64_t smem_opt_in = 0;
+  if (!ensure_dynamic_smem(gemm_tc_kernel, kSmemBytes, smem_opt_in)) return HIF4_ERR_CUDA;
   CUtensorMap tmA, tmB;
   const int64_t upr = K / kUnitElems;
   if (!make_unit_map(&tmA, A, a_rows, upr, BM) || !make_unit_map(&tmB, B, b_rows, upr, BN)) return HIF4_ERR_CUDA;

@@ -345,12 +345,8 @@ bool gemm_tc2_supported(const void* A, const void* B, int64_t M, int64_t N, int6
 
 hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,
                             cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-      return HIF4_ERR_CUDA;
-    attr_set = true;
-  }
+  static uint64_t smem_opt_in = 0;
+  if (!ensure_dynamic_smem(gemm_tc2_kernel, kSmemBytes, smem_opt_in)) return HIF4_ERR_CUDA;
   CUtensorMap tmA, tmB;
   const int64_t upr = K / kUnitElems;
   if (!make_unit_map(&tmA, A, M, upr, kRows) || !make_unit_map(&tmB, B, N, upr, kRows)) return HIF4_ERR_CUDA;

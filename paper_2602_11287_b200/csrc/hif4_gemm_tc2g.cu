@@ -297,12 +297,8 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
 
 hif4_status launch_swapped(const void* A, const void* B, int64_t a_rows, int64_t b_rows, GroupedParams p, int64_t K,
                            cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_tc2g_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-      return HIF4_ERR_CUDA;
-    attr_set = true;
-  }
+  static uint64_t smem_opt_in = 0;
+  if (!ensure_dynamic_smem(gemm_tc2g_kernel, kSmemBytes, smem_opt_in)) return HIF4_ERR_CUDA;
   CUtensorMap tmTok, tmW;
   const int64_t upr = K / kUnitElems;
   if (!make_unit_map(&tmTok, A, a_rows, upr, 128) || !make_unit_map(&tmW, B, b_rows, upr, kWRows)) return HIF4_ERR_CUDA;

@@ -235,12 +235,8 @@ hif4_status launch_gemv_t(const void* B, int64_t upr, const GemvParams& p, cudaS
   constexpr int kRows = 16 * kRowGroups;
   constexpr int smem = 128 + kStages * (kRows * kRawRowBytes + 8 * kTokTiles * kTokChunkBytes) +
                        4 * kChunkWays * kRowGroups * 32 * 4 * kTokTiles * 4 + 16 * kStages + 16;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gemv_kernel<kRowGroups, kTokTiles, kChunkWays>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
-      return HIF4_ERR_CUDA;
-    attr_set = true;
-  }
+  static uint64_t smem_opt_in = 0;
+  if (!ensure_dynamic_smem(gemv_kernel<kRowGroups, kTokTiles, kChunkWays>, smem, smem_opt_in)) return HIF4_ERR_CUDA;
   CUtensorMap tmB;
   if (!make_unit_map(&tmB, B, p.N, upr, kRows)) return HIF4_ERR_CUDA;
   const int64_t blocks = ceil_div64(p.N, kRows);

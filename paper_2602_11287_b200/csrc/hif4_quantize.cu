@@ -14,8 +14,8 @@
 //     multiplied once and the micro-exponent thresholds are taken on maxima of the products;
 //   - fma.rn.bf16x2(t, 4 * 2^-(e8+e16), 128) rounds t's quarter count to nearest-even in the low
 //     mantissa bits (ulp is 1 in [128, 256)); an integer min clamps to 1.75 (and catches Inf).
-// FP32 sources run the same steps in FP32 arithmetic with 16 lanes per unit (lane = one level-3
-// group of 4 elements).
+// FP32 sources run the same steps in FP32 arithmetic with 8 lanes per unit (lane = two level-3
+// groups of 4 elements).
 #include <cuda_bf16.h>
 
 #include "hif4_common.cuh"
@@ -197,37 +197,69 @@ quantize_bf16_kernel(const uint16_t* __restrict__ src, int64_t n_units, int64_t 
 }
 
 // ----------------------------------------------------------------------------- FP32 quantizer
-// 16 lanes per unit, lane k owns level-3 group k (elements 4k..4k+3); lanes 2j, 2j+1 form level-2
-// group j.  Same steps as above in FP32 arithmetic: (1/7) and the reciprocal table are the nearest
-// FP32 values, every product is a single mul.rn.f32.
+// Same steps as above in FP32 arithmetic: (1/7) and the reciprocal table are the nearest FP32 values,
+// every product is a single mul.rn.f32.  One level-3 group (4 elements): micro-exponent from the peak
+// of the products (e8 is passed in), codes as four nibbles in the low 16 bits.
+template <bool kRHA>
+__device__ __forceinline__ uint32_t encode_group_fp32(const uint32_t (&xb)[4], const float (&t)[4], uint32_t p16,
+                                                      uint32_t e8, uint32_t& e16) {
+  e16 = p16 >= 0x40000000u + (e8 << 23);                          // >= 2.0 * 2^e8
+  const float mul = __uint_as_float((129u - (e8 + e16)) << 23);   // 4 * 2^-(e8+e16)
+  uint32_t half = 0;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    uint32_t m;
+    if (!kRHA) {
+      // t * mul is exact (power of two); adding 1.5 * 2^23 rounds it to an integer, nearest-even, in
+      // the low mantissa bits; the integer minimum clamps to 7 and also catches Inf
+      m = min(__float_as_uint(__fmaf_rn(t[e], mul, 12582912.0f)), 0x4B400007u) & 7u;
+    } else {
+      const float q = fminf(__fmul_rn(t[e], mul), 8.0f);
+      const float fl = truncf(q);
+      m = min(static_cast<uint32_t>(fl) + ((q - fl) >= 0.5f ? 1u : 0u), 7u);
+    }
+    half += (m | ((xb[e] >> 28) & 8u)) << (4 * e);
+  }
+  return half;
+}
+
+// 8 lanes per unit.  Lane j loads the 16-byte chunks j and j + 8 of the unit's 256 bytes, i.e. the
+// level-3 groups j and j + 8 (elements 4j..4j+3 and 32+4j..); lanes 2w, 2w+1 together hold the level-2
+// groups w and w + 4.  A warp covers 4 units per pass.
 template <bool kRHA, bool kContig>
 __global__ void __launch_bounds__(kThreads)
 quantize_fp32_kernel(const float* __restrict__ src, int64_t n_units, int64_t upr, int64_t ld_src,
                      uint32_t* __restrict__ dst) {
   const int lane = threadIdx.x & 31;
-  const int k = lane & 15;
+  const int j = lane & 7;
   const int64_t warp = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) >> 5;
-  const int64_t first = warp * (2 * kUnroll) + (lane >> 4);
+  const int64_t first = warp * (4 * kUnroll) + (lane >> 3);
 
-  uint4 v[kUnroll];
+  uint4 va[kUnroll], vb[kUnroll];
 #pragma unroll
   for (int i = 0; i < kUnroll; ++i) {
-    const int64_t u = first + 2 * i;
-    v[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (u < n_units)
-      v[i] = ld_stream(reinterpret_cast<const uint4*>(src + unit_offset<kContig>(u, upr, ld_src) + 4 * k));
+    const int64_t u = first + 4 * i;
+    va[i] = make_uint4(0u, 0u, 0u, 0u);
+    vb[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (u < n_units) {
+      const uint4* p = reinterpret_cast<const uint4*>(src + unit_offset<kContig>(u, upr, ld_src)) + j;
+      va[i] = ld_stream(p);
+      vb[i] = ld_stream(p + 8);
+    }
   }
 
 #pragma unroll
   for (int i = 0; i < kUnroll; ++i) {
-    const int64_t u = first + 2 * i;
-    const uint32_t xb[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
-    uint32_t ab[4];
+    const int64_t u = first + 4 * i;
+    const uint32_t xa[4] = {va[i].x, va[i].y, va[i].z, va[i].w};
+    const uint32_t xb[4] = {vb[i].x, vb[i].y, vb[i].z, vb[i].w};
+    uint32_t aa[4], ab[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) ab[e] = xb[e] & 0x7FFFFFFFu;
-    uint32_t vm = max(max(ab[0], ab[1]), max(ab[2], ab[3]));
-#pragma unroll
-    for (int s = 1; s < 16; s <<= 1) vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, s));
+    for (int e = 0; e < 4; ++e) { aa[e] = xa[e] & 0x7FFFFFFFu; ab[e] = xb[e] & 0x7FFFFFFFu; }
+    uint32_t vm = max(max(max(aa[0], aa[1]), max(aa[2], aa[3])), max(max(ab[0], ab[1]), max(ab[2], ab[3])));
+    vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 1));
+    vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 2));
+    vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 4));
     const bool unit_nan = vm > 0x7F800000u;
 
     const float sf = __fmul_rn(__uint_as_float(vm), __uint_as_float(0x3E124925u));   // (1/7)_FP32
@@ -237,43 +269,44 @@ quantize_fp32_kernel(const float* __restrict__ src, int64_t n_units, int64_t upr
     const uint32_t lut = M == 0 ? 0x3F800000u : M == 1 ? 0x3F4CCCCDu : M == 2 ? 0x3F2AAAABu : 0x3F124925u;
     const float rec = __uint_as_float(lut + (48u << 23) - ((byte >> 2) << 23));
 
-    float t[4];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) t[e] = __fmul_rn(__uint_as_float(ab[e]), rec);
-    const uint32_t p16 = max(max(__float_as_uint(t[0]), __float_as_uint(t[1])),
-                             max(__float_as_uint(t[2]), __float_as_uint(t[3])));
-    const uint32_t p8 = max(p16, __shfl_xor_sync(0xFFFFFFFFu, p16, 1));
-    const uint32_t e8 = p8 >= 0x40800000u;                     // >= 4.0
-    const uint32_t e16 = p16 >= 0x40000000u + (e8 << 23);      // >= 2.0 * 2^e8
-    const float mul = __uint_as_float((129u - (e8 + e16)) << 23);   // 4 * 2^-(e8+e16)
-
-    uint32_t half = 0;
+    float ta[4], tb[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      const float q = fminf(__fmul_rn(t[e], mul), 8.0f);
-      uint32_t m;
-      if (!kRHA) {
-        m = static_cast<uint32_t>(__float2int_rn(q));
-      } else {
-        const float fl = truncf(q);
-        m = static_cast<uint32_t>(fl) + ((q - fl) >= 0.5f ? 1u : 0u);
-      }
-      m = min(m, 7u) | ((xb[e] >> 28) & 8u);
-      half |= m << (4 * e);
+      ta[e] = __fmul_rn(__uint_as_float(aa[e]), rec);
+      tb[e] = __fmul_rn(__uint_as_float(ab[e]), rec);
     }
-    const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, half, 1);
-    uint32_t codes = half | (other << 16);                      // meaningful on even lanes
+    const uint32_t p16a = max(max(__float_as_uint(ta[0]), __float_as_uint(ta[1])),
+                              max(__float_as_uint(ta[2]), __float_as_uint(ta[3])));
+    const uint32_t p16b = max(max(__float_as_uint(tb[0]), __float_as_uint(tb[1])),
+                              max(__float_as_uint(tb[2]), __float_as_uint(tb[3])));
+    // level-2 peaks: this lane's group and its neighbour's
+    const uint32_t e8a = max(p16a, __shfl_xor_sync(0xFFFFFFFFu, p16a, 1)) >= 0x40800000u;    // >= 4.0
+    const uint32_t e8b = max(p16b, __shfl_xor_sync(0xFFFFFFFFu, p16b, 1)) >= 0x40800000u;
+    uint32_t e16a, e16b;
+    const uint32_t ha = encode_group_fp32<kRHA>(xa, ta, p16a, e8a, e16a);
+    const uint32_t hb = encode_group_fp32<kRHA>(xb, tb, p16b, e8b, e16b);
+    // even lane 2w: word w = its four nibbles | the odd neighbour's << 16; same for word w + 4
+    const uint32_t mine = ha | (hb << 16);
+    const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, mine, 1);
+    uint32_t codes_a = (mine & 0xFFFFu) | (other << 16);
+    uint32_t codes_b = (mine >> 16) | (other & 0xFFFF0000u);
 
-    uint32_t meta = (e16 << (16 + k)) | ((k & 1) ? 0u : (e8 << (8 + (k >> 1))));
-#pragma unroll
-    for (int s = 1; s < 16; s <<= 1) meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, s);
+    // E1_16 bits 16 + j and 24 + j; E1_8 bits 8 + w and 12 + w come from the even lanes
+    uint32_t meta = (e16a << (16 + j)) | (e16b << (24 + j));
+    if ((j & 1) == 0) meta |= (e8a << (8 + (j >> 1))) | (e8b << (12 + (j >> 1)));
+    meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 1);
+    meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 2);
+    meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 4);
     meta |= byte;
-    if (unit_nan) { meta = 0xFFu; codes = 0u; }
+    if (unit_nan) { meta = 0xFFu; codes_a = 0u; codes_b = 0u; }
 
     if (u < n_units) {
       uint32_t* out = dst + u * kUnitWords;
-      if ((k & 1) == 0) st_stream(out + 1 + (k >> 1), codes);
-      if (k == 0) st_stream(out, meta);
+      if ((j & 1) == 0) {
+        st_stream(out + 1 + (j >> 1), codes_a);
+        st_stream(out + 5 + (j >> 1), codes_b);
+      }
+      if (j == 0) st_stream(out, meta);
     }
   }
 }
@@ -354,7 +387,7 @@ extern "C" hif4_status hif4_quantize(const void* src, hif4_dtype dt, int64_t row
   const int64_t upr = cols / kUnitElems;
   const int64_t n_units = rows * upr;
   const bool contig = ld_src == cols;
-  const int units_per_block = (kThreads / 32) * kUnroll * (dt == HIF4_BF16 ? 8 : 2);
+  const int units_per_block = (kThreads / 32) * kUnroll * (dt == HIF4_BF16 ? 8 : 4);
   const int64_t blocks = ceil_div64(n_units, units_per_block);
   if (blocks > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
