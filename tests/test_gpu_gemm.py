@@ -288,3 +288,61 @@ def test_weight_streaming_kernel_needs_its_workspace(gemv_path):
     ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
     assert hif4.lib.hif4_gemm(a.data_ptr(), b.data_ptr(), c.data_ptr(), 4, 64, 256, 64, ws.data_ptr(), 1024, None) == 5
     assert hif4.launch_count() == before
+
+
+# ------------------------------------------------------------------ exactness of the in-kernel decoders
+def _exhaustive_units(K):
+    """Rows of K/64 units covering every E6M2 byte below NaN x both values of both micro-exponents x all
+    16 codes at every position parity: row r uses byte r % 255, unit u the micro-exponent pattern u % 4,
+    element i the code (i + r + u) % 16 (so each code meets each (byte, e8, e16) at many positions)."""
+    upr = K // 64
+    rows = 255 * 2
+    A = np.zeros((rows, upr, 36), dtype=np.uint8)
+    for r in range(rows):
+        for u in range(upr):
+            pat = (u + r // 255) % 4
+            meta = (r % 255) | ((0xFF if pat & 1 else 0) << 8) | ((0xFFFF if pat & 2 else 0) << 16)
+            if u % 5 == 4:                       # mixed micro-exponents inside one unit
+                meta = (r % 255) | (0xA5 << 8) | (0x3C5A << 16)
+            A[r, u, 0:4] = np.frombuffer(np.uint32(meta).tobytes(), dtype=np.uint8)
+            codes = (np.arange(64) + r + u) % 16
+            A[r, u, 4:] = (codes[0::2] | (codes[1::2] << 4)).astype(np.uint8)
+    return A
+
+
+def _one_hot_units(K):
+    """K rows; row j decodes to 1.0 at position j and 0 elsewhere (E6M2 = 1.0, code 4 = 1.00)."""
+    upr = K // 64
+    B = np.zeros((K, upr, 36), dtype=np.uint8)
+    B[:, :, 0] = 0xC0
+    for j in range(K):
+        B[j, j // 64, 4 + (j % 64) // 2] = 4 << (4 * (j % 2))
+    return B
+
+
+@pytest.mark.parametrize("path,rows", [(1, 510), (2, 510), (3, 510), (0, 100), (4, 16), (4, 7)])
+def test_every_code_under_every_scale_passes_through_the_gemm_exactly(hif4, path, rows):
+    """C = A * B^T with one-hot rows in B returns the decoded elements of A themselves: each in-kernel
+    decoder (CUDA cores, single CTA, CTA pair, swapped pair for few rows, weight streaming) must give
+    exactly the values of Eq. 2, as A operand and as B operand."""
+    K = 256
+    A_all = _exhaustive_units(K)
+    Bh = _one_hot_units(K)
+    want_all = oracle.dequantize(A_all, oracle.FP32)
+    assert np.array_equal(oracle.dequantize(Bh, oracle.FP32), np.eye(K, dtype=np.float32))
+    hif4.hif4_set_gemm_path(path)
+    try:
+        for start in range(0, A_all.shape[0], rows):
+            A = A_all[start:start + rows]
+            a, b = torch.from_numpy(A).cuda(), torch.from_numpy(Bh).cuda()
+            got = hif4.hif4_gemm(a, b).cpu().numpy()                       # exhaustive units as the A operand
+            assert np.array_equal(got.view(np.uint32) & 0x7FFFFFFF, want_all[start:start + rows].view(np.uint32) & 0x7FFFFFFF)
+            nz = want_all[start:start + rows] != 0                           # sign of zero products is not defined by Eq. 3
+            assert np.array_equal(np.signbit(got)[nz], np.signbit(want_all[start:start + rows])[nz])
+            if path == 4:                                                    # (the streaming kernel takes M <= 16 only)
+                continue
+            got_t = hif4.hif4_gemm(b, a).cpu().numpy()                     # and as the B operand
+            assert np.array_equal(np.abs(got_t.T), np.abs(want_all[start:start + rows]))
+    finally:
+        hif4.hif4_set_gemm_path(0)
+    assert hif4.hif4_last_device_status() == 0
