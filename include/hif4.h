@@ -108,6 +108,20 @@ hif4_status hif4_gemm(const void* A_units, const void* B_units, float* C, int64_
                       int64_t K, int64_t ldc, void* workspace, size_t workspace_bytes,
                       void* stream);
 
+/* hif4_linear -- the W4A4 linear layer in one call (Section IV: every linear layer's activations
+ * are converted to HiF4 before the matrix multiplication): Y = HiF4(X) * W^T, i.e. hif4_quantize of the
+ * activations (Algorithm 1) followed by hif4_gemm with pre-quantized weights (Eq. 3), in stream order.
+ *   X          device, [M, K] of `dt` (BF16 or FP32), row stride ld_x elements, rows 16-byte aligned.
+ *   W_units    device, [N, K/64] units (the weight quantized along K beforehand).
+ *   Y          device, [M, N] FP32, row stride ldy.
+ *   workspace  device scratch of at least hif4_linear_workspace bytes, 256-byte aligned: holds the
+ *              packed activations (and what hif4_gemm needs for this shape).
+ * The result is bit-identical to calling hif4_quantize and hif4_gemm one after the other.  */
+hif4_status hif4_linear_workspace(int64_t M, int64_t N, int64_t K, size_t* bytes);
+hif4_status hif4_linear(const void* X, hif4_dtype dt, int64_t ld_x, const void* W_units, float* Y, int64_t M,
+                        int64_t N, int64_t K, int64_t ldy, hif4_round mode, void* workspace,
+                        size_t workspace_bytes, void* stream);
+
 hif4_status hif4_grouped_gemm_workspace(int num_groups, int64_t total_rows, int64_t N, int64_t K,
                                         size_t* bytes);
 

@@ -24,6 +24,7 @@ EXPORTED_SYMBOLS = [
     "hif4_packed_bytes", "hif4_quantize", "hif4_dequantize", "hif4_gemm_workspace", "hif4_gemm",
     "hif4_grouped_gemm_workspace", "hif4_grouped_gemm", "hif4_last_device_status", "hif4_status_string",
     "hif4_launch_count", "hif4_set_gemm_path", "hif4_grouped_gemm_noalloc", "hif4_grouped_gemm_noalloc_capacity",
+    "hif4_linear", "hif4_linear_workspace",
 ]
 
 
@@ -58,6 +59,10 @@ def _load() -> ctypes.CDLL:
     L.hif4_grouped_gemm_noalloc.argtypes = [vp, vp, vp, vp, ci, i64, i64, i64, i64, vp]
     L.hif4_grouped_gemm_noalloc_capacity.restype = sz
     L.hif4_grouped_gemm_noalloc_capacity.argtypes = []
+    L.hif4_linear_workspace.restype = ci
+    L.hif4_linear_workspace.argtypes = [i64, i64, i64, ctypes.POINTER(sz)]
+    L.hif4_linear.restype = ci
+    L.hif4_linear.argtypes = [vp, ci, i64, vp, vp, i64, i64, i64, i64, ci, vp, sz, vp]
     L.hif4_last_device_status.restype = ci
     L.hif4_last_device_status.argtypes = [vp]
     L.hif4_status_string.restype = ctypes.c_char_p
@@ -166,6 +171,36 @@ def hif4_gemm(a_units: torch.Tensor, b_units: torch.Tensor, out: Optional[torch.
     _check("hif4_gemm", lib.hif4_gemm(a_units.data_ptr(), b_units.data_ptr(), out.data_ptr(), M, N, K, ldc,
                                       workspace.data_ptr() if workspace is not None else None,
                                       workspace.numel() if workspace is not None else 0, _stream(stream)))
+    return out
+
+
+def hif4_linear_workspace(M: int, N: int, K: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check("hif4_linear_workspace", lib.hif4_linear_workspace(M, N, K, ctypes.byref(n)))
+    return int(n.value)
+
+
+def hif4_linear(x: torch.Tensor, w_units: torch.Tensor, out: Optional[torch.Tensor] = None, mode: int = HIF4_RNE,
+                workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Y[M, N] (FP32) = HiF4(X[M, K]) @ W[N, K]^T: activations quantized on the fly (Algorithm 1), weights
+    given as HiF4 units [N, K/64, 36]."""
+    _need_cuda(x, w_units, out, workspace)
+    assert x.dim() == 2 and x.stride(1) == 1 and w_units.dtype == torch.uint8 and w_units.dim() == 3
+    assert w_units.is_contiguous() and w_units.shape[2] == UNIT_BYTES
+    M, K = x.shape
+    N = w_units.shape[0]
+    assert w_units.shape[1] * UNIT_ELEMS == K
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32, device=x.device)
+    assert out.dtype == torch.float32 and out.stride(1) == 1
+    need = hif4_linear_workspace(M, N, K)
+    if workspace is None and need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+    ld_x = x.stride(0) if M > 1 else max(K, x.stride(0))
+    ldy = out.stride(0) if M > 1 else max(N, out.stride(0))
+    _check("hif4_linear", lib.hif4_linear(x.data_ptr(), _dtype_code(x.dtype), ld_x, w_units.data_ptr(), out.data_ptr(),
+                                          M, N, K, ldy, mode, workspace.data_ptr() if workspace is not None else None,
+                                          workspace.numel() if workspace is not None else 0, _stream(stream)))
     return out
 
 

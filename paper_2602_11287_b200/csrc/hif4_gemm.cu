@@ -107,3 +107,35 @@ extern "C" hif4_status hif4_grouped_gemm(const void* A_units, const void* B_unit
   return launch_grouped_gemm_simt(A_units, B_units, C, group_offsets_dev, num_groups, total_rows, N, K, ldc,
                                   st);
 }
+
+// ---------------------------------------------------------------------------------------- hif4_linear
+namespace {
+size_t round256(size_t n) { return (n + 255) / 256 * 256; }
+}  // namespace
+
+extern "C" hif4_status hif4_linear_workspace(int64_t M, int64_t N, int64_t K, size_t* bytes) {
+  if (!bytes) return HIF4_ERR_NULL;
+  size_t gemm_bytes = 0;
+  const hif4_status st = hif4_gemm_workspace(M, N, K, &gemm_bytes);
+  if (st != HIF4_OK) return st;
+  *bytes = round256(hif4_packed_bytes(M, K)) + round256(gemm_bytes);
+  return HIF4_OK;
+}
+
+extern "C" hif4_status hif4_linear(const void* X, hif4_dtype dt, int64_t ld_x, const void* W_units, float* Y,
+                                   int64_t M, int64_t N, int64_t K, int64_t ldy, hif4_round mode, void* workspace,
+                                   size_t workspace_bytes, void* stream) {
+  size_t need = 0;
+  const hif4_status ws = hif4_linear_workspace(M, N, K, &need);
+  if (ws != HIF4_OK) return ws;
+  if (M == 0 || N == 0) return (ldy < N) ? HIF4_ERR_SHAPE : HIF4_OK;
+  if (need > 0 && (!workspace || workspace_bytes < need)) return HIF4_ERR_WORKSPACE;
+  if (need > 0 && !aligned(workspace, 256)) return HIF4_ERR_ALIGN;
+  const size_t x_bytes = round256(hif4_packed_bytes(M, K));
+  uint8_t* x_units = static_cast<uint8_t*>(workspace);
+  if (K > 0) {
+    const hif4_status q = hif4_quantize(X, dt, M, K, ld_x, x_units, mode, stream);
+    if (q != HIF4_OK) return q;
+  }
+  return hif4_gemm(x_units, W_units, Y, M, N, K, ldy, x_units + x_bytes, workspace_bytes - x_bytes, stream);
+}

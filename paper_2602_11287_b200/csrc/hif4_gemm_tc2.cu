@@ -213,15 +213,21 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         tc_fence_after();
         const int row0 = tc.m0 + static_cast<int>(rank) * kRows + q * 32;
 #pragma unroll 1
-        for (int c = 0; c < kPairN / kEpiCols; ++c, ++slabs) {
+        for (int c = 0; c < kPairN / kEpiCols; ++c) {
+          // slabs that lie entirely outside C are neither read nor staged: the two staging buffers
+          // alternate over the slabs that are stored, which is what the wait below counts on
+          const bool stored = row0 < p.M && tc.n0 + c * kEpiCols < p.N;            // same for the whole warp
           uint32_t r[16];
-          tc_ld16(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kPairN + c * kEpiCols, r);
-          tc_wait_ld();
+          if (stored) {
+            tc_ld16(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kPairN + c * kEpiCols, r);
+            tc_wait_ld();
+          }
           if (c == kPairN / kEpiCols - 1) {          // accumulator fully read: hand it back before the stores
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + 8 * acc);
           }
+          if (!stored) continue;
           const uint32_t buf = (slabs & 1u) * kEpiSlabBytes;
           if (lane == 0) bulk_wait_read<1>();        // the store that used this buffer two slabs ago has read it
           __syncwarp();
@@ -230,10 +236,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             sts128(my_row + buf + ((static_cast<uint32_t>(v) ^ sw) << 4), r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
           fence_proxy_async_smem();                  // generic-proxy writes -> visible to the TMA store
           __syncwarp();
-          if (lane == 0 && row0 < p.M && tc.n0 + c * kEpiCols < p.N) {
+          if (lane == 0) {
             tma_store_2d(&tmC, tc.n0 + c * kEpiCols, row0, slab0 + buf);
             bulk_commit();
           }
+          ++slabs;
         }
       }
       if (lane == 0) bulk_wait_all();                // shared memory stays valid until the last store has read it

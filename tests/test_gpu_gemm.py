@@ -205,6 +205,23 @@ def test_tensor_core_kernel_random_units_nan_and_guard_bands(tc_path):
     assert (out[0] == -5.0).all() and (out[M + 1] == -5.0).all() and (out[:, N:] == -5.0).all()
 
 
+def test_cta_pair_kernel_few_columns_in_the_last_tile_repeated(hif4):
+    """A last column tile with 8 valid columns leaves 15 of its 16 staged slabs unused; the staging
+    buffers of the TMA-store epilogue must not be reused while a store still reads them."""
+    hif4.hif4_set_gemm_path(3)
+    try:
+        for (M, N, K) in [(300, 520, 1024), (257, 264, 256), (512, 1032, 512)]:
+            g = torch.Generator(device="cuda"); g.manual_seed(M + N + K)
+            a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
+            b = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
+            C = check_full(hif4, a, b, f"pair kernel {M}x{N}x{K}")
+            for _ in range(20):
+                assert torch.equal(C, hif4.hif4_gemm(a, b)), "runs differ"
+    finally:
+        hif4.hif4_set_gemm_path(0)
+    assert hif4.hif4_last_device_status() == 0
+
+
 def test_tensor_core_kernel_c_rows_not_16_byte_aligned(tc_path):
     """ldc odd and a base that is only 4-byte aligned: the kernels fall back from vector / TMA stores."""
     hif4 = tc_path
@@ -346,3 +363,20 @@ def test_every_code_under_every_scale_passes_through_the_gemm_exactly(hif4, path
     finally:
         hif4.hif4_set_gemm_path(0)
     assert hif4.hif4_last_device_status() == 0
+
+
+@pytest.mark.parametrize("M,N,K,dtype", [(1, 300, 512, torch.bfloat16), (16, 64, 256, torch.float32), (70, 257, 768, torch.bfloat16),
+                                          (300, 520, 1024, torch.bfloat16), (5, 33, 192, torch.bfloat16)])
+def test_linear_is_quantize_then_gemm(hif4, M, N, K, dtype):
+    """hif4_linear (one call for the W4A4 layer) gives the bits of the two separate calls, and those are
+    within tolerance of the FP64 reference on the oracle's encodings."""
+    g = torch.Generator(device="cuda"); g.manual_seed(M + N + K)
+    x = torch.randn(M, K, generator=g, device="cuda").to(dtype)
+    w = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
+    y = hif4.hif4_linear(x, w)
+    xq = hif4.hif4_quantize(x)
+    assert torch.equal(y, hif4.hif4_gemm(xq, w))
+    src = wl.bf16_to_u16_numpy(x) if dtype == torch.bfloat16 else x.cpu().numpy()
+    ref, refabs = oracle.gemm_f64(oracle.quantize(src), w.cpu().numpy(), nthreads=8)
+    assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - ref) <= TOL * refabs + 1e-300)
+    assert hif4.lib.hif4_linear(x.data_ptr(), 0, K, w.data_ptr(), y.data_ptr(), M, N, K, N, 0, None, 0, None) == 5
