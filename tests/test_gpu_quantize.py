@@ -144,3 +144,30 @@ def test_dequantize_strided_output_and_roundtrip(hif4):
     # the "simulated 4-bit" tensor stays close to the source (3-bit significand, shared scales)
     rel = (buf[:, :1088] - t.float()).norm() / t.float().norm()
     assert rel < 0.15
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_quantize_random_bit_patterns(hif4, mode):
+    """Uniformly random BF16 and FP32 bit patterns (every exponent, NaN and Inf included), plus units that
+    mix a narrow range of exponents so that the finite path is exercised as well."""
+    rng = np.random.default_rng(100 + mode)
+    # BF16
+    wild = rng.integers(0, 1 << 16, size=(512, 1024), dtype=np.uint32).astype(np.uint16)
+    expo = rng.integers(100, 150, size=(512, 16, 1), dtype=np.uint32)                  # per unit: base exponent
+    mant = rng.integers(0, 1 << 7, size=(512, 16, 64), dtype=np.uint32)
+    sign = rng.integers(0, 2, size=(512, 16, 64), dtype=np.uint32) << 15
+    spread = rng.integers(0, 7, size=(512, 16, 64), dtype=np.uint32)
+    tame = (sign | ((expo - spread) << 7) | mant).astype(np.uint16).reshape(512, 1024)
+    for bits in (wild, tame):
+        got = _gpu_quantize_bits(hif4, bits, mode)
+        _compare_units(got, oracle.quantize(bits, mode, nthreads=8), f"random bf16 bits mode {mode}")
+    # FP32
+    wild32 = rng.integers(0, 1 << 32, size=(256, 1024), dtype=np.uint64).astype(np.uint32).view(np.float32)
+    expo = rng.integers(90, 160, size=(256, 16, 1), dtype=np.uint32)
+    mant = rng.integers(0, 1 << 23, size=(256, 16, 64), dtype=np.uint32)
+    sign = rng.integers(0, 2, size=(256, 16, 64), dtype=np.uint32) << 31
+    spread = rng.integers(0, 7, size=(256, 16, 64), dtype=np.uint32)
+    tame32 = (sign | ((expo - spread) << 23) | mant).astype(np.uint32).reshape(256, 1024).view(np.float32)
+    for x in (wild32, tame32):
+        got = hif4.hif4_quantize(torch.from_numpy(x.copy()).cuda(), mode).cpu().numpy()
+        _compare_units(got, oracle.quantize(x, mode, nthreads=8), f"random fp32 bits mode {mode}")
