@@ -2,9 +2,9 @@
 // streaming CUDA kernels for sm_100a.  Both are bound by HBM traffic: 2 B (or 4 B) read and
 // 0.5625 B written per element for the quantizer, the reverse for the dequantizer.
 //
-// BF16 quantizer, thread mapping: 4 consecutive lanes own one 64-element unit; lane q loads the
-// 16 bytes of level-2 groups q and q + 4 (elements 8q..8q+7 and 32+8q..) with two 128-bit loads, so
-// a warp covers 8 units per pass and each lane issues 2 * kUnroll loads before it computes.  Algorithm 1 is written in BF16 arithmetic; packed bf16x2 instructions with
+// BF16 quantizer, thread mapping: 2 consecutive lanes own one 64-element unit; lane l loads the
+// 16 bytes of the level-2 groups l, l + 2, l + 4, l + 6 with four 128-bit loads, so a warp covers 16
+// units per pass and each lane issues all its loads before it computes.  Algorithm 1 is written in BF16 arithmetic; packed bf16x2 instructions with
 // round-to-nearest-even are exactly that arithmetic for two elements at a time:
 //   - peak magnitudes are integer maxima of the |x| bit patterns (NaN patterns sort above Inf);
 //   - SF = Vmax * (1/7)_BF16 is one mul.rn.bf16x2; rounding SF to the 3-bit-significand E6M2 byte is
@@ -129,45 +129,48 @@ __device__ __forceinline__ uint32_t encode_group_bf16(uint32_t x0, uint32_t x1, 
   return prmt(g0 * 0x1001u, g1 * 0x1001u, 0x7531u);
 }
 
-// Four consecutive lanes own one unit: lane q loads the 16-byte chunks q and q + 4 of its 128 bytes,
-// i.e. the level-2 groups q and q + 4, so that each load instruction of a warp reads eight 64-byte
-// runs and the per-unit scalar work (scale, reciprocal) is shared by 16 elements.  A warp handles 8
-// units per pass and issues all 2 * kUnroll loads before it computes.
+// Two consecutive lanes own one unit: lane l loads the 16-byte chunks l, l + 2, l + 4, l + 6 of its 128
+// bytes, i.e. the level-2 groups of that parity, so that each load instruction of a warp reads one
+// full 32-byte sector per unit and the per-unit scalar work (scale, reciprocal, metadata) is shared
+// by 32 elements.  A warp handles 16 units per pass and issues all 4 * kUnrollBf16 loads before it computes.
+constexpr int kUnrollBf16 = 2;
+
 template <bool kRHA, bool kContig>
 __global__ void __launch_bounds__(kThreads)
 quantize_bf16_kernel(const uint16_t* __restrict__ src, int64_t n_units, int64_t upr, int64_t ld_src,
                      uint32_t* __restrict__ dst) {
   const int lane = threadIdx.x & 31;
-  const int q = lane & 3;
+  const int l = lane & 1;
   const int64_t warp = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) >> 5;
-  const int64_t first = warp * (8 * kUnroll) + (lane >> 2);
-  // metadata bit weights of this lane's two groups: E1_8 bits 8+q, 12+q; E1_16 bits 16+2q(+1), 24+2q(+1)
-  const uint32_t w8 = 0x100u << q, w16 = 0x10000u << (2 * q);
+  const int64_t first = warp * (16 * kUnrollBf16) + (lane >> 1);
+  // metadata bit weights of this lane's groups g = 2i + l: E1_8 bit 8 + g, E1_16 bits 16 + 2g, 17 + 2g
+  const uint32_t w8 = 0x100u << l, w16 = 0x10000u << (2 * l);
 
-  uint4 va[kUnroll], vb[kUnroll];
+  uint4 v[kUnrollBf16][4];
 #pragma unroll
-  for (int i = 0; i < kUnroll; ++i) {
-    const int64_t u = first + 8 * i;
-    va[i] = make_uint4(0u, 0u, 0u, 0u);
-    vb[i] = make_uint4(0u, 0u, 0u, 0u);
+  for (int i = 0; i < kUnrollBf16; ++i) {
+    const int64_t u = first + 16 * i;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) v[i][c] = make_uint4(0u, 0u, 0u, 0u);
     if (u < n_units) {
-      const uint4* p = reinterpret_cast<const uint4*>(src + unit_offset<kContig>(u, upr, ld_src)) + q;
-      va[i] = ld_stream(p);
-      vb[i] = ld_stream(p + 4);
+      const uint4* p = reinterpret_cast<const uint4*>(src + unit_offset<kContig>(u, upr, ld_src)) + l;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) v[i][c] = ld_stream(p + 2 * c);
     }
   }
 
 #pragma unroll
-  for (int i = 0; i < kUnroll; ++i) {
-    const int64_t u = first + 8 * i;
+  for (int i = 0; i < kUnrollBf16; ++i) {
+    const int64_t u = first + 16 * i;
     // Stage 1: peak magnitude of the unit as an integer maximum of the |x| bit patterns (the group
     // peaks are taken on the products in encode_group_bf16).
     constexpr uint32_t kAbs = 0x7FFF7FFFu;
-    uint32_t vm = umax2(umax2(umax2(va[i].x & kAbs, va[i].y & kAbs), umax2(va[i].z & kAbs, va[i].w & kAbs)),
-                        umax2(umax2(vb[i].x & kAbs, vb[i].y & kAbs), umax2(vb[i].z & kAbs, vb[i].w & kAbs)));
+    uint32_t vm = 0u;
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+      vm = umax2(vm, umax2(umax2(v[i][c].x & kAbs, v[i][c].y & kAbs), umax2(v[i][c].z & kAbs, v[i][c].w & kAbs)));
     vm = hmax_halves(vm);
     vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 1));
-    vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 2));
     const bool unit_nan = vm > 0x7F80u;
 
     // Stage 2: level-1 scale, its reciprocal.
@@ -177,21 +180,28 @@ quantize_bf16_kernel(const uint16_t* __restrict__ src, int64_t n_units, int64_t 
     const uint32_t lut = prmt(0x122B4D80u, 0u, (byte & 3u) | 0x4440u);
     const uint32_t rec2 = (lut + 0x5700u - ((byte & 0xFCu) << 5)) * 0x10001u;
 
-    uint32_t e8a, e16a0, e16a1, e8b, e16b0, e16b1;
-    uint32_t codes_a = encode_group_bf16<kRHA>(va[i].x, va[i].y, va[i].z, va[i].w, rec2, e8a, e16a0, e16a1);
-    uint32_t codes_b = encode_group_bf16<kRHA>(vb[i].x, vb[i].y, vb[i].z, vb[i].w, rec2, e8b, e16b0, e16b1);
-
-    uint32_t meta = (e8a + (e8b << 4)) * w8 + (e16a0 + 2u * e16a1 + ((e16b0 + 2u * e16b1) << 8)) * w16;
+    uint32_t codes[4], m8 = 0u, m16 = 0u;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      uint32_t e8, e16a, e16b;
+      codes[c] = encode_group_bf16<kRHA>(v[i][c].x, v[i][c].y, v[i][c].z, v[i][c].w, rec2, e8, e16a, e16b);
+      m8 += e8 << (2 * c);
+      m16 += (e16a + 2u * e16b) << (4 * c);
+    }
+    uint32_t meta = m8 * w8 + m16 * w16;
     meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 1);
-    meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 2);
     meta |= byte;
-    if (unit_nan) { meta = 0xFFu; codes_a = 0u; codes_b = 0u; }   // NaN unit: E6M2 = NaN, all else zero
+    if (unit_nan) {                                      // NaN unit: E6M2 = NaN, all else zero
+      meta = 0xFFu;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) codes[c] = 0u;
+    }
 
     if (u < n_units) {
       uint32_t* out = dst + u * kUnitWords;
-      st_stream(out + 1 + q, codes_a);
-      st_stream(out + 5 + q, codes_b);
-      if (q == 0) st_stream(out, meta);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) st_stream(out + 1 + 2 * c + l, codes[c]);
+      if (l == 0) st_stream(out, meta);
     }
   }
 }
@@ -387,7 +397,7 @@ extern "C" hif4_status hif4_quantize(const void* src, hif4_dtype dt, int64_t row
   const int64_t upr = cols / kUnitElems;
   const int64_t n_units = rows * upr;
   const bool contig = ld_src == cols;
-  const int units_per_block = (kThreads / 32) * kUnroll * (dt == HIF4_BF16 ? 8 : 4);
+  const int units_per_block = (kThreads / 32) * (dt == HIF4_BF16 ? 16 * kUnrollBf16 : 4 * kUnroll);
   const int64_t blocks = ceil_div64(n_units, units_per_block);
   if (blocks > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
