@@ -14,7 +14,7 @@
 //     multiplied once and the micro-exponent thresholds are taken on maxima of the products;
 //   - fma.rn.bf16x2(t, 4 * 2^-(e8+e16), 128) rounds t's quarter count to nearest-even in the low
 //     mantissa bits (ulp is 1 in [128, 256)); an integer min clamps to 1.75 (and catches Inf).
-// FP32 sources run the same steps in FP32 arithmetic with 8 lanes per unit (lane = two level-3
+// FP32 sources run the same steps in FP32 arithmetic with 4 lanes per unit (lane = four level-3
 // groups of 4 elements).
 #include <cuda_bf16.h>
 
@@ -233,43 +233,46 @@ __device__ __forceinline__ uint32_t encode_group_fp32(const uint32_t (&xb)[4], c
   return half;
 }
 
-// 8 lanes per unit.  Lane j loads the 16-byte chunks j and j + 8 of the unit's 256 bytes, i.e. the
-// level-3 groups j and j + 8 (elements 4j..4j+3 and 32+4j..); lanes 2w, 2w+1 together hold the level-2
-// groups w and w + 4.  A warp covers 4 units per pass.
+// 4 lanes per unit.  Lane l loads the 16-byte chunks l, l + 4, l + 8, l + 12 of the unit's 256 bytes,
+// i.e. the level-3 groups of those numbers (4 elements each); lanes 2w', 2w'+1 together hold the level-2
+// groups w' + 2c (c = 0..3).  A warp covers 8 units per pass.
+constexpr int kUnrollFp32 = 2;
+
 template <bool kRHA, bool kContig>
 __global__ void __launch_bounds__(kThreads)
 quantize_fp32_kernel(const float* __restrict__ src, int64_t n_units, int64_t upr, int64_t ld_src,
                      uint32_t* __restrict__ dst) {
   const int lane = threadIdx.x & 31;
-  const int j = lane & 7;
+  const int l = lane & 3;
   const int64_t warp = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) >> 5;
-  const int64_t first = warp * (4 * kUnroll) + (lane >> 3);
+  const int64_t first = warp * (8 * kUnrollFp32) + (lane >> 2);
 
-  uint4 va[kUnroll], vb[kUnroll];
+  uint4 v[kUnrollFp32][4];
 #pragma unroll
-  for (int i = 0; i < kUnroll; ++i) {
-    const int64_t u = first + 4 * i;
-    va[i] = make_uint4(0u, 0u, 0u, 0u);
-    vb[i] = make_uint4(0u, 0u, 0u, 0u);
+  for (int i = 0; i < kUnrollFp32; ++i) {
+    const int64_t u = first + 8 * i;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) v[i][c] = make_uint4(0u, 0u, 0u, 0u);
     if (u < n_units) {
-      const uint4* p = reinterpret_cast<const uint4*>(src + unit_offset<kContig>(u, upr, ld_src)) + j;
-      va[i] = ld_stream(p);
-      vb[i] = ld_stream(p + 8);
+      const uint4* p = reinterpret_cast<const uint4*>(src + unit_offset<kContig>(u, upr, ld_src)) + l;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) v[i][c] = ld_stream(p + 4 * c);
     }
   }
 
 #pragma unroll
-  for (int i = 0; i < kUnroll; ++i) {
-    const int64_t u = first + 4 * i;
-    const uint32_t xa[4] = {va[i].x, va[i].y, va[i].z, va[i].w};
-    const uint32_t xb[4] = {vb[i].x, vb[i].y, vb[i].z, vb[i].w};
-    uint32_t aa[4], ab[4];
+  for (int i = 0; i < kUnrollFp32; ++i) {
+    const int64_t u = first + 8 * i;
+    uint32_t xb[4][4], ab[4][4];
+    uint32_t vm = 0u;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) { aa[e] = xa[e] & 0x7FFFFFFFu; ab[e] = xb[e] & 0x7FFFFFFFu; }
-    uint32_t vm = max(max(max(aa[0], aa[1]), max(aa[2], aa[3])), max(max(ab[0], ab[1]), max(ab[2], ab[3])));
+    for (int c = 0; c < 4; ++c) {
+      xb[c][0] = v[i][c].x; xb[c][1] = v[i][c].y; xb[c][2] = v[i][c].z; xb[c][3] = v[i][c].w;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) { ab[c][e] = xb[c][e] & 0x7FFFFFFFu; vm = max(vm, ab[c][e]); }
+    }
     vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 1));
     vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 2));
-    vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 4));
     const bool unit_nan = vm > 0x7F800000u;
 
     const float sf = __fmul_rn(__uint_as_float(vm), __uint_as_float(0x3E124925u));   // (1/7)_FP32
@@ -279,44 +282,43 @@ quantize_fp32_kernel(const float* __restrict__ src, int64_t n_units, int64_t upr
     const uint32_t lut = M == 0 ? 0x3F800000u : M == 1 ? 0x3F4CCCCDu : M == 2 ? 0x3F2AAAABu : 0x3F124925u;
     const float rec = __uint_as_float(lut + (48u << 23) - ((byte >> 2) << 23));
 
-    float ta[4], tb[4];
+    uint32_t half[4], meta = 0u;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      ta[e] = __fmul_rn(__uint_as_float(aa[e]), rec);
-      tb[e] = __fmul_rn(__uint_as_float(ab[e]), rec);
+    for (int c = 0; c < 4; ++c) {
+      float t[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) t[e] = __fmul_rn(__uint_as_float(ab[c][e]), rec);
+      const uint32_t p16 = max(max(__float_as_uint(t[0]), __float_as_uint(t[1])),
+                               max(__float_as_uint(t[2]), __float_as_uint(t[3])));
+      // level-2 peak: this lane's level-3 group and its neighbour's
+      const uint32_t e8 = max(p16, __shfl_xor_sync(0xFFFFFFFFu, p16, 1)) >= 0x40800000u;    // >= 4.0
+      uint32_t e16;
+      half[c] = encode_group_fp32<kRHA>(xb[c], t, p16, e8, e16);
+      // level-3 group l + 4c -> E1_16 bit 16 + l + 4c; its level-2 group (l >> 1) + 2c -> E1_8 bit, set by the even lane
+      meta |= e16 << (16 + l + 4 * c);
+      if ((l & 1) == 0) meta |= e8 << (8 + (l >> 1) + 2 * c);
     }
-    const uint32_t p16a = max(max(__float_as_uint(ta[0]), __float_as_uint(ta[1])),
-                              max(__float_as_uint(ta[2]), __float_as_uint(ta[3])));
-    const uint32_t p16b = max(max(__float_as_uint(tb[0]), __float_as_uint(tb[1])),
-                              max(__float_as_uint(tb[2]), __float_as_uint(tb[3])));
-    // level-2 peaks: this lane's group and its neighbour's
-    const uint32_t e8a = max(p16a, __shfl_xor_sync(0xFFFFFFFFu, p16a, 1)) >= 0x40800000u;    // >= 4.0
-    const uint32_t e8b = max(p16b, __shfl_xor_sync(0xFFFFFFFFu, p16b, 1)) >= 0x40800000u;
-    uint32_t e16a, e16b;
-    const uint32_t ha = encode_group_fp32<kRHA>(xa, ta, p16a, e8a, e16a);
-    const uint32_t hb = encode_group_fp32<kRHA>(xb, tb, p16b, e8b, e16b);
-    // even lane 2w: word w = its four nibbles | the odd neighbour's << 16; same for word w + 4
-    const uint32_t mine = ha | (hb << 16);
-    const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, mine, 1);
-    uint32_t codes_a = (mine & 0xFFFFu) | (other << 16);
-    uint32_t codes_b = (mine >> 16) | (other & 0xFFFF0000u);
-
-    // E1_16 bits 16 + j and 24 + j; E1_8 bits 8 + w and 12 + w come from the even lanes
-    uint32_t meta = (e16a << (16 + j)) | (e16b << (24 + j));
-    if ((j & 1) == 0) meta |= (e8a << (8 + (j >> 1))) | (e8b << (12 + (j >> 1)));
+    // even lane: word (l >> 1) + 2c = its four nibbles | the odd neighbour's << 16
+    const uint32_t mine01 = half[0] | (half[1] << 16), mine23 = half[2] | (half[3] << 16);
+    const uint32_t other01 = __shfl_xor_sync(0xFFFFFFFFu, mine01, 1), other23 = __shfl_xor_sync(0xFFFFFFFFu, mine23, 1);
+    uint32_t codes[4] = {(mine01 & 0xFFFFu) | (other01 << 16), (mine01 >> 16) | (other01 & 0xFFFF0000u),
+                         (mine23 & 0xFFFFu) | (other23 << 16), (mine23 >> 16) | (other23 & 0xFFFF0000u)};
     meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 1);
     meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 2);
-    meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 4);
     meta |= byte;
-    if (unit_nan) { meta = 0xFFu; codes_a = 0u; codes_b = 0u; }
+    if (unit_nan) {
+      meta = 0xFFu;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) codes[c] = 0u;
+    }
 
     if (u < n_units) {
       uint32_t* out = dst + u * kUnitWords;
-      if ((j & 1) == 0) {
-        st_stream(out + 1 + (j >> 1), codes_a);
-        st_stream(out + 5 + (j >> 1), codes_b);
+      if ((l & 1) == 0) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) st_stream(out + 1 + (l >> 1) + 2 * c, codes[c]);
       }
-      if (j == 0) st_stream(out, meta);
+      if (l == 0) st_stream(out, meta);
     }
   }
 }
@@ -397,7 +399,7 @@ extern "C" hif4_status hif4_quantize(const void* src, hif4_dtype dt, int64_t row
   const int64_t upr = cols / kUnitElems;
   const int64_t n_units = rows * upr;
   const bool contig = ld_src == cols;
-  const int units_per_block = (kThreads / 32) * (dt == HIF4_BF16 ? 16 * kUnrollBf16 : 4 * kUnroll);
+  const int units_per_block = (kThreads / 32) * (dt == HIF4_BF16 ? 16 * kUnrollBf16 : 8 * kUnrollFp32);
   const int64_t blocks = ceil_div64(n_units, units_per_block);
   if (blocks > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
