@@ -352,15 +352,18 @@ dequantize_kernel(const uint32_t* __restrict__ src, int64_t n_units, int64_t upr
     const uint32_t byte = meta[i] & 0xFFu;
     const uint32_t e8 = (meta[i] >> (8 + j)) & 1u;
     const uint32_t e16a = (meta[i] >> (16 + 2 * j)) & 1u, e16b = (meta[i] >> (17 + 2 * j)) & 1u;
-    const float mant = static_cast<float>(4u + (byte & 3u));
-    // exponent field of 2^(E - 48 - 4 + shift): (byte >> 2) - 52 + 127 + shift
-    const float sa = mant * __uint_as_float(((byte >> 2) + 75u + e8 + e16a) << 23);
-    const float sb = mant * __uint_as_float(((byte >> 2) + 75u + e8 + e16b) << 23);
+    // (4 + M) * 2^(E - 48 - 4 + shift) as FP32 bits: exponent field (byte >> 2) - 52 + 127 + 2 + shift, the
+    // three bits of 4 + M on top of the mantissa (1.00, 1.01, 1.10, 1.11)
+    const uint32_t sbits = (((byte >> 2) + 77u + e8) << 23) | ((byte & 3u) << 21);
+    const float sa = __uint_as_float(sbits + (e16a << 23)), sb = __uint_as_float(sbits + (e16b << 23));
+    // m * s without an integer-to-float conversion: (2^23 + m) * s - 2^23 * s in one fused multiply-add
+    // (the exact product is rounded once, and m * s is representable)
+    const float na = -8388608.0f * sa, nb = -8388608.0f * sb;
     uint32_t bits[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-      const uint32_t c = (word[i] >> (4 * e)) & 0xFu;
-      const float val = static_cast<float>(c & 7u) * (e < 4 ? sa : sb);
+      const uint32_t c = word[i] >> (4 * e);
+      const float val = __fmaf_rn(__uint_as_float((c & 7u) | 0x4B000000u), e < 4 ? sa : sb, e < 4 ? na : nb);
       bits[e] = byte == 0xFFu ? 0x7FC00000u : (__float_as_uint(val) | ((c & 8u) << 28));
     }
     const int64_t off = unit_offset<kContig>(u, upr, ld_dst) + 8 * j;
