@@ -75,17 +75,16 @@ __device__ __forceinline__ PairTile pair_tile(const Gemm2Params& p, int t) {
   return PairTile{mt * kPairM, (t - mt * p.n_tiles) * kPairN};
 }
 
-// Decodes the two units held in raw words L[kOff .. kOff+8] and L[kOff+9 .. kOff+17] into decoded
-// stages 2h and 2h+1.  Returns false when a wait gave up.
-template <int kOff>
-__device__ __forceinline__ bool decode_two_units(const uint32_t (&L)[20], const uint32_t (&chunk_addr)[8], uint32_t lut,
+// Decodes the two units held in raw words W[0..8] and W[9..17] into decoded stages 2h and 2h+1.  Returns
+// false when a wait gave up.
+__device__ __forceinline__ bool decode_two_units(const uint32_t (&W)[18], const uint32_t (&chunk_addr)[8], uint32_t lut,
                                                  const DecodeMul& mul, uint32_t dec_empty0, uint32_t dec_full0_leader,
                                                  uint32_t parity_free, volatile uint32_t* abort_flag) {
 #pragma unroll
   for (int u = 0; u < 2; ++u) {
     // warp-uniform outcome, so that the warp barrier below is never reached by a part of the warp
     if (!__all_sync(0xFFFFFFFFu, mbar_wait(dec_empty0 + 8 * u, parity_free, abort_flag))) return false;
-    decode_unit_balanced(L[kOff + 9 * u], &L[kOff + 9 * u + 1], chunk_addr, u * kDecStageBytes, lut, mul);
+    decode_unit_balanced(W[9 * u], &W[9 * u + 1], chunk_addr, u * kDecStageBytes, lut, mul);
     fence_proxy_async_smem();                  // generic-proxy writes -> visible to the tensor core
     // One remote arrive per warp; the warp barrier orders the other lanes' writes and proxy fences
     // before it.
@@ -308,8 +307,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         // proxy: the proxy fence orders these reads before the release.
         fence_proxy_async_smem();
         mbar_arrive(raw_empty + 8 * s);
-        if (h == 0) ok = decode_two_units<0>(L, chunk_addr, lut, p.mul, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
-        else ok = decode_two_units<2>(L, chunk_addr, lut, p.mul, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
+        // units 2h, 2h+1 start at word 0 (h = 0) or 2 (h = 1) of the loaded window; one copy of the decoder
+        // serves both halves (two copies run side by side cost instruction-cache misses)
+        uint32_t W[18];
+#pragma unroll
+        for (int i = 0; i < 18; ++i) W[i] = h ? L[i + 2] : L[i];
+        ok = decode_two_units(W, chunk_addr, lut, p.mul, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
       }
     }
   }

@@ -91,17 +91,16 @@ __device__ __forceinline__ Unit unit_of(const GroupedParams& p, int u) {
   return r;
 }
 
-// Decodes the two units held in raw words L[kOff..] into decoded stages 2h and 2h+1 (skipped for rows
-// that the tile does not use; the barrier protocol runs either way).
-template <int kOff>
-__device__ __forceinline__ bool decode_two_units_g(const uint32_t (&L)[20], bool active, const uint32_t (&chunk_addr)[8],
+// Decodes the two units held in raw words W[0..8], W[9..17] into decoded stages 2h and 2h+1 (skipped for
+// rows that the tile does not use; the barrier protocol runs either way).
+__device__ __forceinline__ bool decode_two_units_g(const uint32_t (&W)[18], bool active, const uint32_t (&chunk_addr)[8],
                                                    uint32_t lut, const DecodeMul& mul, uint32_t dec_empty0,
                                                    uint32_t dec_full0_leader, uint32_t parity_free,
                                                    volatile uint32_t* abort_flag) {
 #pragma unroll
   for (int u = 0; u < 2; ++u) {
     if (!__all_sync(0xFFFFFFFFu, mbar_wait(dec_empty0 + 8 * u, parity_free, abort_flag))) return false;
-    if (active) decode_unit_balanced(L[kOff + 9 * u], &L[kOff + 9 * u + 1], chunk_addr, u * kDecStageBytes, lut, mul);
+    if (active) decode_unit_balanced(W[9 * u], &W[9 * u + 1], chunk_addr, u * kDecStageBytes, lut, mul);
     fence_proxy_async_smem();
     __syncwarp();
     if ((threadIdx.x & 31) == 0) mbar_arrive_cluster(dec_full0_leader + 8 * u);
@@ -274,8 +273,11 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
         }
         fence_proxy_async_smem();                // reads ordered before the async proxy refills the stage
         mbar_arrive(raw_empty + 8 * s);
-        if (h == 0) ok = decode_two_units_g<0>(L, active, chunk_addr, lut, p.mul, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
-        else ok = decode_two_units_g<2>(L, active, chunk_addr, lut, p.mul, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
+        // one copy of the decoder for both halves: units 2h, 2h+1 start at word 0 or 2 of the window
+        uint32_t W[18];
+#pragma unroll
+        for (int i = 0; i < 18; ++i) W[i] = h ? L[i + 2] : L[i];
+        ok = decode_two_units_g(W, active, chunk_addr, lut, p.mul, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
       }
     }
   }
