@@ -85,6 +85,9 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint
 // stored at position W ^ (n & 1) so that the fragment loads of a quarter-warp hit distinct banks.
 __global__ void __launch_bounds__(128)
 gemv_prepare_tokens_kernel(const uint32_t* __restrict__ A, int M, int m_pad, int64_t upr, uint8_t* __restrict__ tokens) {
+  // the streaming kernel may be scheduled right away: it starts fetching weights and waits for this
+  // grid (griddepcontrol.wait) only before it touches the tokens
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;     // (token n, unit U)
   if (idx >= static_cast<int64_t>(m_pad) * upr) return;
   const int n = static_cast<int>(idx / upr);
@@ -139,7 +142,18 @@ gemv_kernel(const __grid_constant__ CUtensorMap tmB, const GemvParams p) {
   if (warp == kWarps) {
     // ---------------------------------------------------------------- producer
     if (lane == 0) {
-      for (int kc = 0; kc < p.num_kc; ++kc) {
+      // Launched as a programmatic dependent of the token preparation: the weights of the first ring
+      // of stages are requested first, then the preparation grid is waited for, then the tokens follow.
+      const int head = p.num_kc < kStages ? p.num_kc : kStages;
+      for (int kc = 0; kc < head; ++kc) {
+        mbar_expect_tx(full + 8 * kc, kStageBytes);
+        tma_load_2d(smem_base + kc * kStageBytes, &tmB, kc * kRawRowBytes, static_cast<int>(row0), full + 8 * kc);
+      }
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      for (int kc = 0; kc < head; ++kc)
+        bulk_load_1d(smem_base + kc * kStageBytes + kWeightBytes,
+                     p.tokens + static_cast<int64_t>(kc) * p.m_pad * kTokChunkBytes, kTokBytes, full + 8 * kc);
+      for (int kc = head; kc < p.num_kc; ++kc) {
         const uint32_t s = kc % kStages, ph = (kc / kStages) & 1u;
         if (!mbar_wait(empty + 8 * s, ph ^ 1u, abort_flag, 32)) break;
         mbar_expect_tx(full + 8 * s, kStageBytes);
@@ -241,9 +255,22 @@ hif4_status launch_gemv_t(const void* B, int64_t upr, const GemvParams& p, cudaS
   if (!make_unit_map(&tmB, B, p.N, upr, kRows)) return HIF4_ERR_CUDA;
   const int64_t blocks = ceil_div64(p.N, kRows);
   if (blocks > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
-  gemv_kernel<kRowGroups, kTokTiles, kChunkWays><<<static_cast<unsigned>(blocks), (4 * kChunkWays * kRowGroups + 1) * 32, smem, st>>>(tmB, p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(blocks));
+  cfg.blockDim = dim3((4 * kChunkWays * kRowGroups + 1) * 32);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;      // may start while the token preparation still runs
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, gemv_kernel<kRowGroups, kTokTiles, kChunkWays>, tmB, p) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return HIF4_ERR_CUDA;
+  }
   note_launch();
-  return launch_status();
+  return HIF4_OK;
 }
 
 }  // namespace
