@@ -7,7 +7,7 @@
 //      laid out per K = 256 chunk as the B fragments of mma.sync.m16n8k16 want them.
 //   2. gemv_kernel: one CTA owns 16 * kRowGroups weight rows and the whole K range.  A producer warp
 //      streams, per K = 256 chunk, the CTA's packed weight rows (one 2-D TMA box, 144 bytes per row) and
-//      the tokens' chunk (one bulk copy, L2-resident) through an 8-stage ring.  Consumer warp (rg, ks)
+//      the tokens' chunk (one bulk copy, L2-resident) through a 4- or 8-stage ring.  Consumer warp (rg, ks)
 //      owns 16 weight rows and unit ks of every kChunkWays-th chunk (8 or 16 K slices per row group, so
 //      that even a narrow problem has enough warps in flight to hide the decode latency): lane (g, q) reads the metadata word and code words
 //      2q, 2q+1 of rows g and g+8, decodes them in registers straight into the A fragments (weights are
@@ -22,7 +22,6 @@
 namespace hif4 {
 namespace {
 
-constexpr int kStages = 8;
 constexpr int kTokChunkBytes = 512;                  // one token, K = 256, BF16
 
 struct GemvParams {
@@ -109,7 +108,7 @@ gemv_prepare_tokens_kernel(const uint32_t* __restrict__ A, int M, int m_pad, int
   }
 }
 
-template <int kRowGroups, int kTokTiles, int kChunkWays>
+template <int kRowGroups, int kTokTiles, int kChunkWays, int kStages>
 __global__ void __launch_bounds__((4 * kChunkWays * kRowGroups + 1) * 32)
 gemv_kernel(const __grid_constant__ CUtensorMap tmB, const GemvParams p) {
   constexpr int kWarps = 4 * kChunkWays * kRowGroups;              // consumer warps
@@ -244,13 +243,13 @@ gemv_kernel(const __grid_constant__ CUtensorMap tmB, const GemvParams p) {
   }
 }
 
-template <int kRowGroups, int kTokTiles, int kChunkWays>
+template <int kRowGroups, int kTokTiles, int kChunkWays, int kStages>
 hif4_status launch_gemv_t(const void* B, int64_t upr, const GemvParams& p, cudaStream_t st) {
   constexpr int kRows = 16 * kRowGroups;
   constexpr int smem = 128 + kStages * (kRows * kRawRowBytes + 8 * kTokTiles * kTokChunkBytes) +
                        4 * kChunkWays * kRowGroups * 32 * 4 * kTokTiles * 4 + 16 * kStages + 16;
   static uint64_t smem_opt_in = 0;
-  if (!ensure_dynamic_smem(gemv_kernel<kRowGroups, kTokTiles, kChunkWays>, smem, smem_opt_in)) return HIF4_ERR_CUDA;
+  if (!ensure_dynamic_smem(gemv_kernel<kRowGroups, kTokTiles, kChunkWays, kStages>, smem, smem_opt_in)) return HIF4_ERR_CUDA;
   CUtensorMap tmB;
   if (!make_unit_map(&tmB, B, p.N, upr, kRows)) return HIF4_ERR_CUDA;
   const int64_t blocks = ceil_div64(p.N, kRows);
@@ -265,7 +264,7 @@ hif4_status launch_gemv_t(const void* B, int64_t upr, const GemvParams& p, cudaS
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, gemv_kernel<kRowGroups, kTokTiles, kChunkWays>, tmB, p) != cudaSuccess) {
+  if (cudaLaunchKernelEx(&cfg, gemv_kernel<kRowGroups, kTokTiles, kChunkWays, kStages>, tmB, p) != cudaSuccess) {
     (void)cudaGetLastError();
     return HIF4_ERR_CUDA;
   }
@@ -302,8 +301,8 @@ hif4_status launch_gemv(const void* A, const void* B, float* C, int64_t M, int64
   // 16 weight rows per CTA with 16 K slices for narrow problems (few CTAs, so each needs many warps),
   // 32 rows with 4 K slices per row group once that still gives every SM two CTAs
   const bool wide = N >= 64ll * sm_count();
-  if (p.m_pad == 8) return wide ? launch_gemv_t<2, 1, 1>(B, upr, p, st) : launch_gemv_t<1, 1, 4>(B, upr, p, st);
-  return wide ? launch_gemv_t<2, 2, 1>(B, upr, p, st) : launch_gemv_t<1, 2, 4>(B, upr, p, st);
+  if (p.m_pad == 8) return wide ? launch_gemv_t<2, 1, 1, 4>(B, upr, p, st) : launch_gemv_t<1, 1, 4, 8>(B, upr, p, st);
+  return wide ? launch_gemv_t<2, 2, 1, 4>(B, upr, p, st) : launch_gemv_t<1, 2, 4, 8>(B, upr, p, st);
 }
 
 }  // namespace hif4
