@@ -307,7 +307,7 @@ def measure_reference_points(dev):
 
 def measure_e2e(hif4, dev, weights, world, args):
     """Same step through the public API with HOST buffers: pinned BF16 activations copied in, FP32
-    results copied out, every step."""
+    results copied out, every step; copies and kernels overlap on three streams."""
     host_x, dev_x, host_c, dev_c, dev_q = {}, {}, {}, {}, {}
     for (M, K, N, name) in SHAPES:
         if (M, K) not in host_x:
@@ -320,17 +320,50 @@ def measure_e2e(hif4, dev, weights, world, args):
     h2d = sum(t.numel() * 2 for t in host_x.values())
     d2h = sum(t.numel() * 4 for t in host_c.values())
 
+    # Three streams: pinned activations in, kernels, results out.  Events order each buffer's reuse: the
+    # kernels of a shape wait for its activations, the copy-out waits for its GEMM, the next step's GEMM
+    # waits until the previous result has left, the next step's copy-in until the quantizers have read.
+    compute = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    in_ready = {k: torch.cuda.Event() for k in host_x}
+    x_consumed = {k: torch.cuda.Event() for k in host_x}
+    c_ready = {k: torch.cuda.Event() for k in host_c}
+    c_left = {k: torch.cuda.Event() for k in host_c}
+    last_user = {}
+    for (M, K, N, name) in SHAPES:
+        last_user[(M, K)] = (M, K, N)
+    state = {"first": True}
+
     def step():
-        for key, t in host_x.items():
-            dev_x[key].copy_(t, non_blocking=True)
+        with torch.cuda.stream(s_in):
+            for key, t in host_x.items():
+                if not state["first"]:
+                    s_in.wait_event(x_consumed[key])
+                dev_x[key].copy_(t, non_blocking=True)
+                in_ready[key].record(s_in)
         for (M, K, N, name) in SHAPES:
+            compute.wait_event(in_ready[(M, K)])
             hif4.hif4_quantize(dev_x[(M, K)], out=dev_q[(M, K, N)])
+            if last_user[(M, K)] == (M, K, N):
+                x_consumed[(M, K)].record(compute)
+            if not state["first"]:
+                compute.wait_event(c_left[(M, K, N)])
             hif4.hif4_gemm(dev_q[(M, K, N)], weights[(K, N)], out=dev_c[(M, K, N)], workspace=ws)
-            host_c[(M, K, N)].copy_(dev_c[(M, K, N)], non_blocking=True)
+            c_ready[(M, K, N)].record(compute)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(c_ready[(M, K, N)])
+                host_c[(M, K, N)].copy_(dev_c[(M, K, N)], non_blocking=True)
+                c_left[(M, K, N)].record(s_out)
+        state["first"] = False
+
+    def join():
+        for ev in c_left.values():
+            compute.wait_event(ev)
 
     steps = max(3, min(args.steps, 10))
     for _ in range(2):
         step()
+    join()
     torch.cuda.synchronize()
     if world > 1:
         import torch.distributed as dist
@@ -339,6 +372,7 @@ def measure_e2e(hif4, dev, weights, world, args):
     s.record()
     for _ in range(steps):
         step()
+    join()                                   # the step is over when its last result has reached the host
     e.record()
     torch.cuda.synchronize()
     ms = s.elapsed_time(e) / steps
