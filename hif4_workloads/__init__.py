@@ -121,7 +121,7 @@ def moe_routing(tokens: int = MOE_TOKENS, experts: int = MOE_EXPERTS, topk: int 
     logp = torch.empty(experts, device=device, dtype=torch.float64)
     logp[perm] = logp_by_rank
     u = torch.rand(tokens, experts, generator=g, device=device, dtype=torch.float64).clamp_(1e-300, 1.0)
-    gumbel = -torch.log(-torch.log(u).clamp_min(1e-300))
+    gumbel = -torch.log((-torch.log(u)).clamp_min(1e-300))
     choice = torch.topk(logp.unsqueeze(0) + gumbel, topk, dim=1).indices      # [tokens, topk]
     flat_expert = choice.reshape(-1)
     flat_token = torch.arange(tokens, device=device).repeat_interleave(topk)

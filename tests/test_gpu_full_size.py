@@ -100,6 +100,7 @@ def test_moe_layer_grouped_full_size(hif4):
     counts = r["counts"].cpu().numpy()
     total = int(off[-1])
     assert total == wl.MOE_TOKENS * wl.MOE_TOPK and len(counts) == wl.MOE_EXPERTS
+    assert (counts > 0).sum() >= 250 and counts.max() > 2000 and np.median(counts) < 80, "Zipf-shaped expert loads"
     off_h = off.cpu().numpy()
     order = np.argsort(counts)
     picks = [int(order[-1]), int(order[0]), int(order[len(order) // 2]), int(order[-2]), int(order[len(order) // 4])]
