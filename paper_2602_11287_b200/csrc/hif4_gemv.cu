@@ -1,19 +1,19 @@
 // Decode-shaped HiF4 GEMM (M <= 16 tokens): C = A * B^T with the weight matrix B streamed once from
-// HBM.  The problem is bound by the 0.5625 bytes per weight element that have to cross the memory
-// bus, so the kernel is organised around keeping many TMA copies of packed weight rows in flight,
-// and the few tokens are prepared once.
+// HBM.  The few tokens are decoded once; the work per weight element is the register decode, so the
+// kernel is organised around decoding with as few instructions per element as possible and around
+// giving every SM the same number of weight rows.
 //
 //   1. gemv_prepare_tokens_kernel decodes the M rows of A (Eq. 2, exact BF16) into a small workspace
 //      laid out per K = 256 chunk as the B fragments of mma.sync.m16n8k16 want them.
-//   2. gemv_kernel: one CTA owns 16 * kRowGroups weight rows and the whole K range.  A producer warp
-//      streams, per K = 256 chunk, the CTA's packed weight rows (one 2-D TMA box, 144 bytes per row) and
-//      the tokens' chunk (one bulk copy, L2-resident) through a 4- or 8-stage ring.  Consumer warp (rg, ks)
-//      owns 16 weight rows and unit ks of every kChunkWays-th chunk (8 or 16 K slices per row group, so
-//      that even a narrow problem has enough warps in flight to hide the decode latency): lane (g, q) reads the metadata word and code words
-//      2q, 2q+1 of rows g and g+8, decodes them in registers straight into the A fragments (weights are
-//      the 16-row MMA operand), reads the matching token fragments from shared memory and issues four
-//      BF16 MMAs with FP32 accumulators.  Inside a unit the K order is permuted the same way on both
-//      operands.  The K slices are summed through shared memory in a fixed order.
+//   2. gemv_kernel: one CTA per SM owns a contiguous run of 8-row blocks of B (the runs differ by at
+//      most one block) and the whole K range.  A producer warp streams, per K = 256 chunk, the CTA's
+//      packed weight rows (one 2-D TMA box, 144 bytes per row) and the tokens' chunk (one bulk copy,
+//      L2-resident) through a ring of stages.  Consumer warp (pair, way) owns two 8-row blocks (the 16
+//      rows of the MMA's weight operand) and every `ways`-th chunk.  Lane (g, q) owns unit q of the
+//      chunk for rows g and g + 8: it reads the two 36-byte units, prepares the unit's scales once, and
+//      decodes word after word straight into the A fragments (k slots 2q, 2q+1, 2q+8, 2q+9 of every MMA
+//      come from unit q on both operands, so the K order is permuted the same way on both sides).
+//      The K slices of a pair are summed through shared memory in a fixed order.
 // Results are deterministic (no atomics).  Every mbarrier wait is bounded.
 #include "hif4_common.cuh"
 #include "hif4_gemm_internal.cuh"
@@ -23,16 +23,26 @@ namespace hif4 {
 namespace {
 
 constexpr int kTokChunkBytes = 512;                  // one token, K = 256, BF16
+constexpr int kTileChunkBytes = 8 * kTokChunkBytes;  // eight tokens (one MMA n-tile), K = 256
+constexpr int kBlockRows = 8;                        // granule of the row partition
+constexpr int kBlockBytes = kBlockRows * kRawRowBytes;   // 1152 = 9 * 128
+constexpr int kMaxBlocks = 16;                       // 8-row blocks per CTA (TMA box of up to 128 rows)
+constexpr int kMaxStages = 16;
+constexpr int kGemvWarps = 24;                       // consumer warps per CTA
+constexpr int kRingBudget = 176 * 1024;              // bytes of shared memory given to the ring of stages
 
 struct GemvParams {
   const uint32_t* A;        // [M, K/64] units (tokens)
-  uint8_t* tokens;          // workspace: [K/256][m_pad][512 B]
+  uint8_t* tokens;          // workspace: [K/256][tiles][8 words][8 tokens][4 units][16 B]
   float* C;
   int64_t ldc;
   int M;
-  int m_pad;                // 8 or 16
   int64_t N;
   int num_kc;               // K / 256
+  int num_blocks;           // ceil(N / 8)
+  int max_blocks;           // 8-row blocks of the largest CTA; the others have one fewer
+  int stages;
+  DecodeMul mul;
   unsigned int* error_word;
 };
 
@@ -80,8 +90,8 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint
                : "memory");
 }
 
-// Token workspace: chunk kc, token n: 512 bytes = 4 units x 8 words x 16 bytes, the 16-byte group of word W
-// stored at position W ^ (n & 1) so that the fragment loads of a quarter-warp hit distinct banks.
+// Token workspace: chunk kc, n-tile t, word W: 512 bytes = 8 tokens x 4 units x 16 bytes, so that the 32
+// lanes (token g, unit q) of a warp read one contiguous, conflict-free line per word.
 __global__ void __launch_bounds__(128)
 gemv_prepare_tokens_kernel(const uint32_t* __restrict__ A, int M, int m_pad, int64_t upr, uint8_t* __restrict__ tokens) {
   // the streaming kernel may be scheduled right away: it starts fetching weights and waits for this
@@ -91,10 +101,11 @@ gemv_prepare_tokens_kernel(const uint32_t* __restrict__ A, int M, int m_pad, int
   if (idx >= static_cast<int64_t>(m_pad) * upr) return;
   const int n = static_cast<int>(idx / upr);
   const int64_t U = idx - static_cast<int64_t>(n) * upr;
-  uint4* dst = reinterpret_cast<uint4*>(tokens + ((U >> 2) * m_pad + n) * kTokChunkBytes + (U & 3) * 128);
+  const int tiles = m_pad >> 3;
+  uint8_t* dst = tokens + (((U >> 2) * tiles + (n >> 3)) * 8) * kTokChunkBytes + ((n & 7) * 4 + (U & 3)) * 16;
   if (n >= M) {
 #pragma unroll
-    for (int W = 0; W < 8; ++W) dst[W] = make_uint4(0u, 0u, 0u, 0u);
+    for (int W = 0; W < 8; ++W) *reinterpret_cast<uint4*>(dst + W * kTokChunkBytes) = make_uint4(0u, 0u, 0u, 0u);
     return;
   }
   const uint32_t* unit = A + (static_cast<int64_t>(n) * upr + U) * kUnitWords;
@@ -103,135 +114,196 @@ gemv_prepare_tokens_kernel(const uint32_t* __restrict__ A, int M, int m_pad, int
   for (int W = 0; W < 8; W += 2) {
     uint32_t r[8];
     decode_two_words(meta, W, __ldg(unit + 1 + W), __ldg(unit + 2 + W), r);
-    dst[W ^ (n & 1)] = make_uint4(r[0], r[1], r[2], r[3]);
-    dst[(W + 1) ^ (n & 1)] = make_uint4(r[4], r[5], r[6], r[7]);
+    *reinterpret_cast<uint4*>(dst + W * kTokChunkBytes) = make_uint4(r[0], r[1], r[2], r[3]);
+    *reinterpret_cast<uint4*>(dst + (W + 1) * kTokChunkBytes) = make_uint4(r[4], r[5], r[6], r[7]);
   }
 }
 
-template <int kRowGroups, int kTokTiles, int kChunkWays, int kStages>
-__global__ void __launch_bounds__((4 * kChunkWays * kRowGroups + 1) * 32)
-gemv_kernel(const __grid_constant__ CUtensorMap tmB, const GemvParams p) {
-  constexpr int kWarps = 4 * kChunkWays * kRowGroups;              // consumer warps
-  constexpr int kRows = 16 * kRowGroups;
-  constexpr int kWeightBytes = kRows * kRawRowBytes;
-  constexpr int kTokBytes = 8 * kTokTiles * kTokChunkBytes;
-  constexpr int kStageBytes = kWeightBytes + kTokBytes;            // multiples of 128
-  constexpr int kRedBytes = kWarps * 32 * 4 * kTokTiles * 4;       // partial accumulators of every consumer warp
+// Per-unit part of the weight decode: the BF16 bits of E6M2 / 4 in both halves, the constant that is
+// OR-ed into every element pair (128.0, or NaN for a NaN unit, Eq. 2), and E1_8[j] + E1_16[2j] /
+// E1_16[2j+1] for all eight words as two-bit fields of the low / high half.
+struct UnitPrep {
+  uint32_t base2, or_k, sum;
+};
+__device__ __forceinline__ UnitPrep prepare_unit(uint32_t meta, uint32_t lut) {
+  UnitPrep u;
+  const uint32_t byte = meta & 0xFFu;
+  u.or_k = byte == 0xFFu ? 0x7FC07FC0u : 0x43004300u;
+  u.base2 = byte * 0x00200020u + 0x26802680u;                       // ((byte + 308) << 5) in both halves
+  u.sum = (((meta >> 16) & 0x5555u) | ((meta >> 1) & 0x55550000u)) + lds32(lut + ((meta >> 6) & 0x3FCu));
+  return u;
+}
+// Word j of the unit -> four bf16x2 registers holding elements (0,4), (1,5), (2,6), (3,7) of level-2
+// group j.  Left shifts and most additions are written as multiply-adds with run-time multipliers so
+// that they issue on the multiply-add pipe instead of the integer/logic pipe.
+__device__ __forceinline__ void decode_word(const UnitPrep& u, int j, uint32_t wj, const DecodeMul& k, uint32_t (&r)[4]) {
+  const uint32_t f = ((u.sum >> (2 * j)) * k.m128) & 0x01800180u;    // field j at the exponent's low bits
+  const uint32_t Sa = f * k.one + u.base2;                          // (S_lo, S_hi), S = E6M2 * 2^(e8 + e16 - 2)
+  const uint32_t Sb = Sa - 0x02000200u;                             // S / 16
+  const uint32_t Oa = Sa * k.one + 0x83808380u;                     // -128 S
+  const uint32_t Ob = Sa * k.one + 0x81808180u;                     // -8 S
+  const uint32_t wh = wj >> 8;
+  r[0] = fma_bf16x2((wj & 0x00070007u) | u.or_k, Sa, Oa) ^ ((wj * k.m4096) & 0x80008000u);
+  r[1] = fma_bf16x2((wj & 0x00700070u) | u.or_k, Sb, Ob) ^ ((wj * k.m256) & 0x80008000u);
+  r[2] = fma_bf16x2((wh & 0x00070007u) | u.or_k, Sa, Oa) ^ ((wj * k.m16) & 0x80008000u);
+  r[3] = fma_bf16x2((wh & 0x00700070u) | u.or_k, Sb, Ob) ^ (wj & 0x80008000u);
+}
+
+// A parity wait cannot tell a barrier that is one phase behind from one that is done, so a consumer
+// first waits until the producer has announced the chunk it wants for that stage (the producer only
+// announces it after every reader of the stage's previous chunk has arrived).  Bounded like mbar_wait.
+__device__ __forceinline__ bool wait_announced(const volatile int* slot, int kc, volatile uint32_t* abort_flag) {
+  if (*slot >= kc) return true;
+  const uint64_t t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (*slot >= kc) return true;
+    __nanosleep(64);
+    if ((it & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > kWaitBudgetNs) {
+        *abort_flag = 1u;
+        return false;
+      }
+    }
+  }
+}
+
+// Shared memory: [spread table 1 KB][partial sums][barriers, abort word, announced chunks: 384 B][ring of stages, 128-byte aligned]
+template <int kTokTiles>
+__global__ void __launch_bounds__((kGemvWarps + 1) * 32, 1)
+gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__ CUtensorMap tm_short, const GemvParams p) {
+  constexpr int kTokBytes = kTokTiles * kTileChunkBytes;
+  constexpr int kRedBytes = kGemvWarps * 32 * 4 * kTokTiles * 4;     // partial accumulators of every consumer warp
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 127u) & ~127u;
-  const uint32_t bar_base = smem_base + kStages * kStageBytes + kRedBytes;
-  const uint32_t full = bar_base, empty = bar_base + 8 * kStages;
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
-  float* red = reinterpret_cast<float*>(gen_base + kStages * kStageBytes);
-  volatile uint32_t* abort_flag =
-      reinterpret_cast<volatile uint32_t*>(gen_base + kStages * kStageBytes + kRedBytes + 16 * kStages);
+  const uint32_t lut = smem_base;
+  float* red = reinterpret_cast<float*>(gen_base + 1024);
+  const uint32_t bar_base = smem_base + 1024 + kRedBytes;
+  const uint32_t full = bar_base, empty = bar_base + 8 * kMaxStages;
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(gen_base + 1024 + kRedBytes + 16 * kMaxStages);
+  volatile int* announced = reinterpret_cast<volatile int*>(gen_base + 1024 + kRedBytes + 16 * kMaxStages + 16);   // chunk in each stage
+  const uint32_t ring = bar_base + 384;
+  const uint32_t w_bytes_max = static_cast<uint32_t>(p.max_blocks) * kBlockBytes;
+  const uint32_t stage_bytes = w_bytes_max + kTokBytes;
+
+  // this CTA's run of 8-row blocks
+  const int64_t blk_begin = static_cast<int64_t>(blockIdx.x) * p.num_blocks / gridDim.x;
+  const int nblk = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * p.num_blocks / gridDim.x - blk_begin);
+  const int npairs = (nblk + 1) >> 1;
+  const int ways = kGemvWarps / npairs;              // >= 1: npairs <= kMaxBlocks / 2
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int64_t row0 = static_cast<int64_t>(blockIdx.x) * kRows;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < p.stages; ++s) {
       mbar_init(full + 8 * s, 1);
-      mbar_init(empty + 8 * s, 4 * kRowGroups);          // the warps that read one chunk
+      mbar_init(empty + 8 * s, npairs);                // the warps that read one chunk
+      announced[s] = -1;
     }
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (threadIdx.x < 256) reinterpret_cast<uint32_t*>(gen_base)[threadIdx.x] = spread_e8_entry(threadIdx.x);
   __syncthreads();
 
-  if (warp == kWarps) {
+  if (warp == kGemvWarps) {
     // ---------------------------------------------------------------- producer
     if (lane == 0) {
+      const CUtensorMap* map = nblk == p.max_blocks ? &tm_full : &tm_short;
+      const uint32_t tx = static_cast<uint32_t>(nblk) * kBlockBytes + kTokBytes;
+      const int row0 = static_cast<int>(blk_begin * kBlockRows);
       // Launched as a programmatic dependent of the token preparation: the weights of the first ring
       // of stages are requested first, then the preparation grid is waited for, then the tokens follow.
-      const int head = p.num_kc < kStages ? p.num_kc : kStages;
+      const int head = p.num_kc < p.stages ? p.num_kc : p.stages;
       for (int kc = 0; kc < head; ++kc) {
-        mbar_expect_tx(full + 8 * kc, kStageBytes);
-        tma_load_2d(smem_base + kc * kStageBytes, &tmB, kc * kRawRowBytes, static_cast<int>(row0), full + 8 * kc);
+        announced[kc] = kc;
+        mbar_expect_tx(full + 8 * kc, tx);
+        tma_load_2d(ring + kc * stage_bytes, map, kc * kRawRowBytes, row0, full + 8 * kc);
       }
       asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int kc = 0; kc < head; ++kc)
-        bulk_load_1d(smem_base + kc * kStageBytes + kWeightBytes,
-                     p.tokens + static_cast<int64_t>(kc) * p.m_pad * kTokChunkBytes, kTokBytes, full + 8 * kc);
+        bulk_load_1d(ring + kc * stage_bytes + w_bytes_max, p.tokens + static_cast<int64_t>(kc) * kTokBytes, kTokBytes,
+                     full + 8 * kc);
+      uint32_t s = 0, ph = 1;                          // stage and phase of chunk `head`
       for (int kc = head; kc < p.num_kc; ++kc) {
-        const uint32_t s = kc % kStages, ph = (kc / kStages) & 1u;
         if (!mbar_wait(empty + 8 * s, ph ^ 1u, abort_flag, 32)) break;
-        mbar_expect_tx(full + 8 * s, kStageBytes);
-        const uint32_t dst = smem_base + s * kStageBytes;
-        tma_load_2d(dst, &tmB, kc * kRawRowBytes, static_cast<int>(row0), full + 8 * s);
-        bulk_load_1d(dst + kWeightBytes, p.tokens + static_cast<int64_t>(kc) * p.m_pad * kTokChunkBytes, kTokBytes,
-                     full + 8 * s);
+        announced[s] = kc;
+        __threadfence_block();
+        mbar_expect_tx(full + 8 * s, tx);
+        const uint32_t dst = ring + s * stage_bytes;
+        tma_load_2d(dst, map, kc * kRawRowBytes, row0, full + 8 * s);
+        bulk_load_1d(dst + w_bytes_max, p.tokens + static_cast<int64_t>(kc) * kTokBytes, kTokBytes, full + 8 * s);
+        if (++s == static_cast<uint32_t>(p.stages)) { s = 0; ph ^= 1u; }
       }
     }
   } else {
     // ---------------------------------------------------------------- consumers: 16 weight rows x one K slice per warp
-    // row group, K slice: unit (slice & 3) of the chunks kc = slice / 4 (mod kChunkWays)
-    const int rg = warp % kRowGroups, slice = warp / kRowGroups, ks = slice & 3, way = slice >> 2;
+    const int pair = warp % npairs, way = warp / npairs;
+    const bool active = way < ways;
+    const bool has_hi = 2 * pair + 1 < nblk;           // the pair's second block exists
     const int g = lane >> 2, q = lane & 3;
-    // two accumulator sets per token tile, so that consecutive MMAs do not wait on one another
-    float acc[kTokTiles][4], acc2[kTokTiles][4];
+    float acc[kTokTiles][4];
 #pragma unroll
     for (int t = 0; t < kTokTiles; ++t)
 #pragma unroll
-      for (int i = 0; i < 4; ++i) acc[t][i] = acc2[t][i] = 0.0f;
-    const uint32_t w_off0 = static_cast<uint32_t>(16 * rg + g) * kRawRowBytes + ks * kUnitBytes;   // MMA row g
-    const uint32_t w_off1 = w_off0 + 8 * kRawRowBytes;                                               // MMA row g + 8
-    // token g (and g + 8): words 2q and 2q+1 of unit ks, 16-byte groups swizzled by the token's parity
-    const uint32_t t_base = kWeightBytes + static_cast<uint32_t>(g) * kTokChunkBytes + ks * 128;
-    const uint32_t t_lo = t_base + ((static_cast<uint32_t>(2 * q) ^ (g & 1u)) << 4);
-    const uint32_t t_hi = t_base + ((static_cast<uint32_t>(2 * q + 1) ^ (g & 1u)) << 4);
-    bool ok = true;
-    for (int kc = way; kc < p.num_kc && ok; kc += kChunkWays) {
-      const uint32_t s = kc % kStages, ph = (kc / kStages) & 1u;
-      if (!(ok = __all_sync(0xFFFFFFFFu, mbar_wait(full + 8 * s, ph, abort_flag)))) break;
-      const uint32_t st = smem_base + s * kStageBytes;
-      uint32_t a[8], b[8];
-      const uint32_t r0 = st + w_off0, r1 = st + w_off1;
-      const uint32_t m0 = lds32(r0), w00 = lds32(r0 + 4 + 8 * q), w01 = lds32(r0 + 8 + 8 * q);
-      const uint32_t m1 = lds32(r1), w10 = lds32(r1 + 4 + 8 * q), w11 = lds32(r1 + 8 + 8 * q);
-      uint4 x[kTokTiles], y[kTokTiles];
+      for (int i = 0; i < 4; ++i) acc[t][i] = 0.0f;
+    const uint32_t off_lo = static_cast<uint32_t>(16 * pair + g) * kRawRowBytes + q * kUnitBytes;   // MMA row g
+    const uint32_t off_hi = off_lo + 8 * kRawRowBytes;                                                // MMA row g + 8
+    const uint32_t off_tok = w_bytes_max + static_cast<uint32_t>(lane) * 16;
+    if (active) {
+      uint32_t s = static_cast<uint32_t>(way % p.stages), ph = static_cast<uint32_t>(way / p.stages) & 1u;
+      const uint32_t s_step = static_cast<uint32_t>(ways % p.stages), ph_step = static_cast<uint32_t>(ways / p.stages);
+      bool ok = true;
+      for (int kc = way; kc < p.num_kc; kc += ways) {
+        if (!(ok = __all_sync(0xFFFFFFFFu, wait_announced(announced + s, kc, abort_flag) &&
+                                               mbar_wait(full + 8 * s, ph, abort_flag))))
+          break;
+        const uint32_t st = ring + s * stage_bytes;
+        const uint32_t ml = lds32(st + off_lo), mh = has_hi ? lds32(st + off_hi) : 0u;
+        const UnitPrep ul = prepare_unit(ml, lut), uh = prepare_unit(mh, lut);
+        // a short loop rather than eight unrolled words: the body stays small enough for the instruction cache
+#pragma unroll 2
+        for (int j = 0; j < 8; ++j) {
+          uint4 x[kTokTiles];
 #pragma unroll
-      for (int t = 0; t < kTokTiles; ++t) {
-        x[t] = lds128(st + t_lo + t * 8 * kTokChunkBytes);
-        y[t] = lds128(st + t_hi + t * 8 * kTokChunkBytes);
-      }
-      fence_proxy_async_smem();                  // reads done before the async proxy refills the stage
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty + 8 * s);
-      decode_two_words(m0, 2 * q, w00, w01, a);
-      decode_two_words(m1, 2 * q, w10, w11, b);
+          for (int t = 0; t < kTokTiles; ++t) x[t] = lds128(st + off_tok + (t * 8 + j) * kTokChunkBytes);
+          uint32_t a[4], b[4] = {0u, 0u, 0u, 0u};
+          decode_word(ul, j, lds32(st + off_lo + 4 + 4 * j), p.mul, a);
+          if (has_hi) decode_word(uh, j, lds32(st + off_hi + 4 + 4 * j), p.mul, b);
 #pragma unroll
-      for (int t = 0; t < kTokTiles; ++t) {
-        mma_bf16_16816(acc[t], a[0], b[0], a[1], b[1], x[t].x, x[t].y);
-        mma_bf16_16816(acc2[t], a[2], b[2], a[3], b[3], x[t].z, x[t].w);
-        mma_bf16_16816(acc[t], a[4], b[4], a[5], b[5], y[t].x, y[t].y);
-        mma_bf16_16816(acc2[t], a[6], b[6], a[7], b[7], y[t].z, y[t].w);
+          for (int t = 0; t < kTokTiles; ++t) {
+            mma_bf16_16816(acc[t], a[0], b[0], a[1], b[1], x[t].x, x[t].y);
+            mma_bf16_16816(acc[t], a[2], b[2], a[3], b[3], x[t].z, x[t].w);
+          }
+        }
+        fence_proxy_async_smem();                  // reads done before the async proxy refills the stage
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty + 8 * s);
+        s += s_step; ph += ph_step;
+        if (s >= static_cast<uint32_t>(p.stages)) { s -= p.stages; ++ph; }
+        ph &= 1u;
       }
     }
-#pragma unroll
-    for (int t = 0; t < kTokTiles; ++t)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) acc[t][i] += acc2[t][i];
-    // Sum the K slices of every row group in a fixed order, then store.
+    // Sum the K slices of every pair in a fixed order, then store.
     float* mine = red + (static_cast<size_t>(warp) * 32 + lane) * (4 * kTokTiles);
 #pragma unroll
     for (int t = 0; t < kTokTiles; ++t)
 #pragma unroll
       for (int i = 0; i < 4; ++i) mine[4 * t + i] = acc[t][i];
-    asm volatile("bar.sync 1, %0;" ::"n"(kWarps * 32) : "memory");     // consumer warps only
-    if (slice == 0 && !*abort_flag) {
+    asm volatile("bar.sync 1, %0;" ::"n"(kGemvWarps * 32) : "memory");     // consumer warps only
+    if (way == 0 && !*abort_flag) {
       // acc[t]: {row g: tokens 2q, 2q+1; row g+8: tokens 2q, 2q+1} (+ 8 t)
-      const int64_t n0 = row0 + 16 * rg + g;
+      const int64_t n0 = (blk_begin + 2 * pair) * kBlockRows + g;
 #pragma unroll
       for (int t = 0; t < kTokTiles; ++t)
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           float v = acc[t][i];
-#pragma unroll
-          for (int k = 1; k < 4 * kChunkWays; ++k)
-            v += red[(static_cast<size_t>(k * kRowGroups + rg) * 32 + lane) * (4 * kTokTiles) + 4 * t + i];
+          for (int k = 1; k < ways; ++k)
+            v += red[(static_cast<size_t>(k * npairs + pair) * 32 + lane) * (4 * kTokTiles) + 4 * t + i];
           const int tok = 8 * t + 2 * q + (i & 1);
           const int64_t n = n0 + (i >> 1) * 8;
-          if (tok < p.M && n < p.N) p.C[static_cast<int64_t>(tok) * p.ldc + n] = v;
+          if (tok < p.M && n < p.N && ((i >> 1) == 0 || has_hi)) p.C[static_cast<int64_t>(tok) * p.ldc + n] = v;
         }
     }
   }
@@ -243,20 +315,29 @@ gemv_kernel(const __grid_constant__ CUtensorMap tmB, const GemvParams p) {
   }
 }
 
-template <int kRowGroups, int kTokTiles, int kChunkWays, int kStages>
-hif4_status launch_gemv_t(const void* B, int64_t upr, const GemvParams& p, cudaStream_t st) {
-  constexpr int kRows = 16 * kRowGroups;
-  constexpr int smem = 128 + kStages * (kRows * kRawRowBytes + 8 * kTokTiles * kTokChunkBytes) +
-                       4 * kChunkWays * kRowGroups * 32 * 4 * kTokTiles * 4 + 16 * kStages + 16;
+template <int kTokTiles>
+hif4_status launch_gemv_t(const void* B, int64_t upr, GemvParams p, cudaStream_t st) {
+  constexpr int kTokBytes = kTokTiles * kTileChunkBytes;
+  constexpr int kFixed = 128 + 1024 + kGemvWarps * 32 * 4 * kTokTiles * 4 + 384;
+  // One CTA per SM (several rounds of them when a CTA would get more than kMaxBlocks blocks).
+  const int64_t sms = sm_count();
+  const int64_t rounds = ceil_div64(p.num_blocks, sms * kMaxBlocks);
+  const int64_t grid = p.num_blocks < sms * rounds ? p.num_blocks : sms * rounds;
+  if (grid > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
+  p.max_blocks = static_cast<int>(ceil_div64(p.num_blocks, grid));
+  const int stage_bytes = p.max_blocks * kBlockBytes + kTokBytes;
+  p.stages = kRingBudget / stage_bytes;
+  if (p.stages > kMaxStages) p.stages = kMaxStages;
+  if (p.stages > p.num_kc) p.stages = p.num_kc;
+  const int smem = kFixed + p.stages * stage_bytes;
   static uint64_t smem_opt_in = 0;
-  if (!ensure_dynamic_smem(gemv_kernel<kRowGroups, kTokTiles, kChunkWays, kStages>, smem, smem_opt_in)) return HIF4_ERR_CUDA;
-  CUtensorMap tmB;
-  if (!make_unit_map(&tmB, B, p.N, upr, kRows)) return HIF4_ERR_CUDA;
-  const int64_t blocks = ceil_div64(p.N, kRows);
-  if (blocks > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
+  if (!ensure_dynamic_smem(gemv_kernel<kTokTiles>, kFixed + kRingBudget, smem_opt_in)) return HIF4_ERR_CUDA;
+  CUtensorMap tm_full, tm_short;
+  if (!make_unit_map(&tm_full, B, p.N, upr, p.max_blocks * kBlockRows)) return HIF4_ERR_CUDA;
+  if (!make_unit_map(&tm_short, B, p.N, upr, (p.max_blocks > 1 ? p.max_blocks - 1 : 1) * kBlockRows)) return HIF4_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(blocks));
-  cfg.blockDim = dim3((4 * kChunkWays * kRowGroups + 1) * 32);
+  cfg.gridDim = dim3(static_cast<unsigned>(grid));
+  cfg.blockDim = dim3((kGemvWarps + 1) * 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -264,7 +345,7 @@ hif4_status launch_gemv_t(const void* B, int64_t upr, const GemvParams& p, cudaS
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, gemv_kernel<kRowGroups, kTokTiles, kChunkWays, kStages>, tmB, p) != cudaSuccess) {
+  if (cudaLaunchKernelEx(&cfg, gemv_kernel<kTokTiles>, tm_full, tm_short, p) != cudaSuccess) {
     (void)cudaGetLastError();
     return HIF4_ERR_CUDA;
   }
@@ -289,20 +370,20 @@ hif4_status launch_gemv(const void* A, const void* B, float* C, int64_t M, int64
   GemvParams p{};
   p.A = static_cast<const uint32_t*>(A);
   p.tokens = static_cast<uint8_t*>(workspace);
-  p.C = C; p.ldc = ldc; p.M = static_cast<int>(M); p.m_pad = M <= 8 ? 8 : 16; p.N = N;
+  p.C = C; p.ldc = ldc; p.M = static_cast<int>(M); p.N = N;
   p.num_kc = static_cast<int>(K / 256);
+  if (ceil_div64(N, kBlockRows) > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
+  p.num_blocks = static_cast<int>(ceil_div64(N, kBlockRows));
+  p.mul = make_decode_mul();
   p.error_word = device_error_word();
   if (!p.error_word) return HIF4_ERR_CUDA;
+  const int m_pad = M <= 8 ? 8 : 16;
   const int64_t upr = K / kUnitElems;
-  const int64_t prep = static_cast<int64_t>(p.m_pad) * upr;
-  gemv_prepare_tokens_kernel<<<static_cast<unsigned>(ceil_div64(prep, 128)), 128, 0, st>>>(p.A, p.M, p.m_pad, upr, p.tokens);
+  const int64_t prep = static_cast<int64_t>(m_pad) * upr;
+  gemv_prepare_tokens_kernel<<<static_cast<unsigned>(ceil_div64(prep, 128)), 128, 0, st>>>(p.A, p.M, m_pad, upr, p.tokens);
   note_launch();
   if (cudaGetLastError() != cudaSuccess) return HIF4_ERR_CUDA;
-  // 16 weight rows per CTA with 16 K slices for narrow problems (few CTAs, so each needs many warps),
-  // 32 rows with 4 K slices per row group once that still gives every SM two CTAs
-  const bool wide = N >= 64ll * sm_count();
-  if (p.m_pad == 8) return wide ? launch_gemv_t<2, 1, 1, 4>(B, upr, p, st) : launch_gemv_t<1, 1, 4, 8>(B, upr, p, st);
-  return wide ? launch_gemv_t<2, 2, 1, 4>(B, upr, p, st) : launch_gemv_t<1, 2, 4, 8>(B, upr, p, st);
+  return m_pad == 8 ? launch_gemv_t<1>(B, upr, p, st) : launch_gemv_t<2>(B, upr, p, st);
 }
 
 }  // namespace hif4

@@ -262,7 +262,8 @@ def gemv_path(hif4):
 
 
 @pytest.mark.parametrize("M,N,K", [(1, 1, 256), (1, 64, 256), (2, 33, 512), (7, 200, 1024), (8, 4096, 256), (9, 130, 768),
-                                   (16, 1000, 2304), (16, 64, 4096), (5, 9475, 256), (3, 31, 5120), (12, 77, 14336)])
+                                   (16, 1000, 2304), (16, 64, 4096), (5, 9475, 256), (3, 31, 5120), (12, 77, 14336),
+                                   (1, 40003, 256), (16, 2376, 1024), (10, 1192, 512), (4, 19000, 256)])
 def test_weight_streaming_kernel_full_compare(gemv_path, M, N, K):
     hif4 = gemv_path
     g = torch.Generator(device="cuda"); g.manual_seed(M * 11 + N)
