@@ -148,9 +148,15 @@ def run_cuda(args):
     torch.cuda.synchronize()
 
     stream = torch.cuda.current_stream()
+    # Step order: M=1 linears, two prefill linears, M=16 linears, two prefill linears -- more than the
+    # 126 MB of L2 is touched between two uses of any weight matrix (M=1 and M=16 share theirs).
+    big = [sh for sh in SHAPES if sh[0] >= 4096]
+    groups = [[sh for sh in SHAPES if sh[0] == 1], big[:2], [sh for sh in SHAPES if sh[0] == 16], big[2:]]
+    small = groups[0] + groups[2]                       # decode-shaped: microseconds per kernel, launch-bound
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
-    def step(events=None):
-        for (M, K, N, name) in SHAPES:
+    def run_shapes(shapes, events=None):
+        for (M, K, N, name) in shapes:
             if events is not None:
                 e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
                 e0.record(stream)
@@ -169,9 +175,33 @@ def run_cuda(args):
     sampler = ClockSampler(local_rank)
     sampler.start()
     for _ in range(max(args.warmup, 3)):
-        step()
+        run_shapes(SHAPES)
     barrier()
 
+    # The launches of the decode-shaped linears are captured once into two CUDA graphs (M=1, M=16) and
+    # replayed every step (their kernels run a few microseconds each, so launch gaps would dominate);
+    # the four prefill linears are launched directly, with events around them for the roofline.
+    graphs, graph_launches = {}, 0
+    if not args.no_graph:
+        for gi in (0, 2):
+            n0 = hif4.launch_count()
+            graphs[gi] = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graphs[gi]):
+                run_shapes(groups[gi])
+            graph_launches += hif4.launch_count() - n0
+        torch.cuda.synchronize()
+
+    def step(events=None):
+        for gi, shapes in enumerate(groups):
+            if gi in graphs:
+                graphs[gi].replay()
+            elif gi in (0, 2):
+                run_shapes(shapes)
+            else:
+                run_shapes(shapes, events)
+
+    step()
+    barrier()
     events = []
     launches0 = hif4.launch_count()
     barrier()
@@ -183,18 +213,28 @@ def run_cuda(args):
     t_end.record(stream)
     barrier()
     host_t1 = time.time()
-    launches = hif4.launch_count() - launches0
+    launches = hif4.launch_count() - launches0 + graph_launches * args.steps
     clocks = sampler.stop(host_t0, host_t1)
     elapsed_ms = dp.max_over_ranks(t_start.elapsed_time(t_end), dev)
     status = hif4.hif4_last_device_status()
     if status != 0:
         raise SystemExit(f"device status {status}: {hif4.status_string(status)}")
 
+    # per-kernel times of the decode-shaped linears: a separate pass with events around every call and
+    # L2 flushed (a 256 MB write) before each linear
+    small_events = []
+    for _ in range(20):
+        for sh in small:
+            flush.zero_()
+            run_shapes([sh], small_events)
+    torch.cuda.synchronize()
+    events += small_events
+
     step_flops = sum(flops(M, K, N) for (M, K, N, _) in SHAPES)
     ms_per_step = elapsed_ms / args.steps
     value = dp.job_throughput(step_flops, world, ms_per_step * 1e-3) / 1e12
 
-    # ---- per-kernel times inside the timed region
+    # ---- per-kernel times (prefill shapes: inside the timed region; decode shapes: the pass above)
     per_shape = {}
     for (shape, e0, e1, e2) in events:
         d = per_shape.setdefault(shape, [0.0, 0.0, 0])
@@ -227,7 +267,11 @@ def run_cuda(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16 x bf16 -> f32 (HiF4 decoded exactly to bf16)",
         "data": "synthetic",
         "config": {"workload": WORKLOAD, "weights": "pre-quantized to HiF4, resident",
-                   "l2": "no flush: a step touches ~0.9 GB (> 126 MB L2) before it returns to any tensor",
+                   "l2": "no flush: the step order (M=1 linears, two prefill linears, M=16 linears, two prefill linears) "
+                         "touches > 126 MB (L2) between two uses of any tensor; per_shape rows with M <= 16 come from "
+                         "a separate pass that writes 256 MB before each linear",
+                   "launch": ("decode-shaped linears replayed from two CUDA graphs per step, prefill linears launched directly"
+                              if graphs else "every kernel launched directly"),
                    "parallelism": f"dp{world} (independent token batches, no collective)"},
         "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "per_shape": table,
     }
@@ -523,6 +567,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch the decode-shaped linears directly instead of replaying a CUDA graph")
     ap.add_argument("--gemm-path", type=int, default=0, help="with --case: kernel selection, see hif4_set_gemm_path")
     ap.add_argument("--case", default=None,
                     help="run one kernel a few times instead of the benchmark (for ncu captures): "
