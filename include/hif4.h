@@ -60,7 +60,11 @@ typedef enum {
   HIF4_ERR_UNSUPPORTED = 8     /* valid request that this build does not implement             */
 } hif4_status;
 
-typedef enum { HIF4_BF16 = 0, HIF4_FP32 = 1 } hif4_dtype;
+/* HIF4_FP16 is a source type only (hif4_quantize, hif4_linear): Section II-B applies the conversion to
+ * "other high-precision formats, such as FP32 and FP16"; FP16 arithmetic cannot hold the reciprocal of an
+ * E6M2 scale (up to 2^48), so FP16 elements are widened exactly to FP32 and Algorithm 1 runs in FP32
+ * arithmetic.  hif4_dequantize returns HIF4_ERR_DTYPE for it (HiF4's range exceeds FP16's).  */
+typedef enum { HIF4_BF16 = 0, HIF4_FP32 = 1, HIF4_FP16 = 2 } hif4_dtype;
 
 /* Rounding used where Algorithm 1 rounds to E6M2 and to S1P2 ("round-half-to-even or
  * round-half-away-from-zero", Section II-B).  Products inside the algorithm always round to
@@ -78,7 +82,7 @@ size_t hif4_packed_bytes(int64_t rows, int64_t cols);
  *              storage gives the fastest stores).  Fully overwritten.
  *   mode       HIF4_RNE or HIF4_RHA.
  * The working precision of the algorithm is that of the source type (BF16 arithmetic for BF16
- * input, FP32 arithmetic for FP32 input).  A unit holding a NaN becomes the canonical NaN unit
+ * input, FP32 arithmetic for FP32 and FP16 input).  A unit holding a NaN becomes the canonical NaN unit
  * (meta 0x000000FF, codes 0).  rows == 0 or cols == 0 is a no-op returning HIF4_OK.  */
 hif4_status hif4_quantize(const void* src, hif4_dtype dt, int64_t rows, int64_t cols,
                           int64_t ld_src, void* dst_units, hif4_round mode, void* stream);

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhif4.so")
 
 UNIT_ELEMS, UNIT_BYTES = 64, 36
-HIF4_BF16, HIF4_FP32 = 0, 1
+HIF4_BF16, HIF4_FP32, HIF4_FP16 = 0, 1, 2
 HIF4_RNE, HIF4_RHA = 0, 1
 HIF4_OK = 0
 
@@ -97,7 +97,9 @@ def _dtype_code(dt: torch.dtype) -> int:
         return HIF4_BF16
     if dt == torch.float32:
         return HIF4_FP32
-    raise TypeError(f"HiF4 conversion takes bfloat16 or float32, not {dt}")
+    if dt == torch.float16:
+        return HIF4_FP16                                  # source type only: the library rejects it as a destination
+    raise TypeError(f"HiF4 conversion takes bfloat16, float32 or (as a source) float16, not {dt}")
 
 
 def _need_cuda(*tensors: torch.Tensor) -> None:

@@ -17,6 +17,7 @@
 // FP32 sources run the same steps in FP32 arithmetic with 4 lanes per unit (lane = four level-3
 // groups of 4 elements).
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "hif4_common.cuh"
 
@@ -233,14 +234,25 @@ __device__ __forceinline__ uint32_t encode_group_fp32(const uint32_t (&xb)[4], c
   return half;
 }
 
-// 4 lanes per unit.  Lane l loads the 16-byte chunks l, l + 4, l + 8, l + 12 of the unit's 256 bytes,
-// i.e. the level-3 groups of those numbers (4 elements each); lanes 2w', 2w'+1 together hold the level-2
+// 4 lanes per unit.  Lane l loads the level-3 groups l, l + 4, l + 8, l + 12 (4 elements each: 16-byte chunks
+// of an FP32 unit, 8-byte chunks of an FP16 unit); lanes 2w', 2w'+1 together hold the level-2
 // groups w' + 2c (c = 0..3).  A warp covers 8 units per pass.
 constexpr int kUnrollFp32 = 2;
 
-template <bool kRHA, bool kContig>
+// Four consecutive source elements (one level-3 group) as FP32 bit patterns.  FP16 elements are widened,
+// which is exact, so an FP16 tensor encodes like the FP32 tensor of the same values.
+__device__ __forceinline__ uint4 load_group_fp32(const float* p) { return ld_stream(reinterpret_cast<const uint4*>(p)); }
+__device__ __forceinline__ uint4 load_group_fp32(const __half* p) {
+  uint2 h;
+  asm volatile("ld.global.cs.v2.u32 {%0,%1}, [%2];" : "=r"(h.x), "=r"(h.y) : "l"(p));
+  const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&h.x));
+  const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&h.y));
+  return make_uint4(__float_as_uint(lo.x), __float_as_uint(lo.y), __float_as_uint(hi.x), __float_as_uint(hi.y));
+}
+
+template <bool kRHA, bool kContig, typename Src>
 __global__ void __launch_bounds__(kThreads)
-quantize_fp32_kernel(const float* __restrict__ src, int64_t n_units, int64_t upr, int64_t ld_src,
+quantize_fp32_kernel(const Src* __restrict__ src, int64_t n_units, int64_t upr, int64_t ld_src,
                      uint32_t* __restrict__ dst) {
   const int lane = threadIdx.x & 31;
   const int l = lane & 3;
@@ -254,9 +266,9 @@ quantize_fp32_kernel(const float* __restrict__ src, int64_t n_units, int64_t upr
 #pragma unroll
     for (int c = 0; c < 4; ++c) v[i][c] = make_uint4(0u, 0u, 0u, 0u);
     if (u < n_units) {
-      const uint4* p = reinterpret_cast<const uint4*>(src + unit_offset<kContig>(u, upr, ld_src)) + l;
+      const Src* p = src + unit_offset<kContig>(u, upr, ld_src) + 4 * l;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) v[i][c] = ld_stream(p + 4 * c);
+      for (int c = 0; c < 4; ++c) v[i][c] = load_group_fp32(p + 16 * c);
     }
   }
 
@@ -384,6 +396,15 @@ dequantize_kernel(const uint32_t* __restrict__ src, int64_t n_units, int64_t upr
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
+template <typename Src>
+void launch_quantize_fp32(const Src* x, bool rha, bool contig, dim3 grid, cudaStream_t st, int64_t n_units, int64_t upr,
+                          int64_t ld_src, uint32_t* dst) {
+  if (!rha && contig) quantize_fp32_kernel<false, true, Src><<<grid, kThreads, 0, st>>>(x, n_units, upr, ld_src, dst);
+  else if (!rha) quantize_fp32_kernel<false, false, Src><<<grid, kThreads, 0, st>>>(x, n_units, upr, ld_src, dst);
+  else if (contig) quantize_fp32_kernel<true, true, Src><<<grid, kThreads, 0, st>>>(x, n_units, upr, ld_src, dst);
+  else quantize_fp32_kernel<true, false, Src><<<grid, kThreads, 0, st>>>(x, n_units, upr, ld_src, dst);
+}
+
 }  // namespace
 }  // namespace hif4
 
@@ -391,12 +412,12 @@ using namespace hif4;
 
 extern "C" hif4_status hif4_quantize(const void* src, hif4_dtype dt, int64_t rows, int64_t cols,
                                      int64_t ld_src, void* dst_units, hif4_round mode, void* stream) {
-  if (dt != HIF4_BF16 && dt != HIF4_FP32) return HIF4_ERR_DTYPE;
+  if (dt != HIF4_BF16 && dt != HIF4_FP32 && dt != HIF4_FP16) return HIF4_ERR_DTYPE;
   if (mode != HIF4_RNE && mode != HIF4_RHA) return HIF4_ERR_DTYPE;
   if (rows < 0 || cols < 0 || cols % kUnitElems != 0 || ld_src < cols) return HIF4_ERR_SHAPE;
   if (rows == 0 || cols == 0) return HIF4_OK;
   if (!src || !dst_units) return HIF4_ERR_NULL;
-  const size_t esz = dt == HIF4_BF16 ? 2 : 4;
+  const size_t esz = dt == HIF4_FP32 ? 4 : 2;
   if (!aligned(src, 16) || (static_cast<size_t>(ld_src) * esz) % 16 != 0 || !aligned(dst_units, 4))
     return HIF4_ERR_ALIGN;
   const int64_t upr = cols / kUnitElems;
@@ -408,19 +429,18 @@ extern "C" hif4_status hif4_quantize(const void* src, hif4_dtype dt, int64_t row
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint32_t* dst = static_cast<uint32_t*>(dst_units);
   const dim3 grid(static_cast<unsigned>(blocks));
-#define HIF4_LAUNCH_Q(KERNEL, T)                                                                 \
-  do {                                                                                           \
-    if (mode == HIF4_RNE) {                                                                      \
-      if (contig) KERNEL<false, true><<<grid, kThreads, 0, st>>>(static_cast<const T*>(src), n_units, upr, ld_src, dst); \
-      else KERNEL<false, false><<<grid, kThreads, 0, st>>>(static_cast<const T*>(src), n_units, upr, ld_src, dst);       \
-    } else {                                                                                     \
-      if (contig) KERNEL<true, true><<<grid, kThreads, 0, st>>>(static_cast<const T*>(src), n_units, upr, ld_src, dst);  \
-      else KERNEL<true, false><<<grid, kThreads, 0, st>>>(static_cast<const T*>(src), n_units, upr, ld_src, dst);        \
-    }                                                                                            \
-  } while (0)
-  if (dt == HIF4_BF16) HIF4_LAUNCH_Q(quantize_bf16_kernel, uint16_t);
-  else HIF4_LAUNCH_Q(quantize_fp32_kernel, float);
-#undef HIF4_LAUNCH_Q
+  const bool rha = mode == HIF4_RHA;
+  if (dt == HIF4_BF16) {
+    const uint16_t* x = static_cast<const uint16_t*>(src);
+    if (!rha && contig) quantize_bf16_kernel<false, true><<<grid, kThreads, 0, st>>>(x, n_units, upr, ld_src, dst);
+    else if (!rha) quantize_bf16_kernel<false, false><<<grid, kThreads, 0, st>>>(x, n_units, upr, ld_src, dst);
+    else if (contig) quantize_bf16_kernel<true, true><<<grid, kThreads, 0, st>>>(x, n_units, upr, ld_src, dst);
+    else quantize_bf16_kernel<true, false><<<grid, kThreads, 0, st>>>(x, n_units, upr, ld_src, dst);
+  } else if (dt == HIF4_FP32) {
+    launch_quantize_fp32(static_cast<const float*>(src), rha, contig, grid, st, n_units, upr, ld_src, dst);
+  } else {
+    launch_quantize_fp32(static_cast<const __half*>(src), rha, contig, grid, st, n_units, upr, ld_src, dst);
+  }
   note_launch();
   return launch_status();
 }

@@ -106,7 +106,7 @@ def test_quantize_empty_and_bad_arguments(hif4):
         hif4.hif4_quantize(torch.zeros(2, 64, dtype=torch.bfloat16, device="cuda"), mode=7)
     assert ei.value.code == 4
     with pytest.raises(TypeError):
-        hif4.hif4_quantize(torch.zeros(2, 64, dtype=torch.float16, device="cuda"))
+        hif4.hif4_quantize(torch.zeros(2, 64, dtype=torch.float64, device="cuda"))
     with pytest.raises(ValueError):
         hif4.hif4_quantize(torch.zeros(2, 64, dtype=torch.bfloat16))
     assert hif4.hif4_last_device_status() == 0
@@ -171,3 +171,37 @@ def test_quantize_random_bit_patterns(hif4, mode):
     for x in (wild32, tame32):
         got = hif4.hif4_quantize(torch.from_numpy(x.copy()).cuda(), mode).cpu().numpy()
         _compare_units(got, oracle.quantize(x, mode, nthreads=8), f"random fp32 bits mode {mode}")
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_quantize_fp16_source(hif4, mode):
+    """FP16 sources (widened exactly to FP32, then Algorithm 1 in FP32 arithmetic): every FP16 bit pattern
+    (subnormals, Inf and NaN included), units of a narrow exponent range, a strided source, and the one-call
+    linear layer on FP16 activations."""
+    rng = np.random.default_rng(300 + mode)
+    every = np.arange(1 << 16, dtype=np.uint16)
+    rng.shuffle(every)
+    wild = every.reshape(64, 1024).view(np.float16)
+    expo = rng.integers(3, 28, size=(256, 16, 1), dtype=np.uint32)
+    mant = rng.integers(0, 1 << 10, size=(256, 16, 64), dtype=np.uint32)
+    sign = rng.integers(0, 2, size=(256, 16, 64), dtype=np.uint32) << 15
+    spread = rng.integers(0, 4, size=(256, 16, 64), dtype=np.uint32)
+    tame = (sign | (np.maximum(expo - spread, 0) << 10) | mant).astype(np.uint16).reshape(256, 1024).view(np.float16)
+    for x in (wild, tame):
+        got = hif4.hif4_quantize(torch.from_numpy(x.copy()).cuda(), mode).cpu().numpy()
+        _compare_units(got, oracle.quantize(x, mode, nthreads=8), f"fp16 bits mode {mode}")
+    # strided source: columns [64, 64 + 320) of a wider tensor, guard band around the output
+    wide = torch.from_numpy(tame.copy()).cuda()
+    view = wide[:37, 64:384]
+    out = torch.full((39, 5, 36), 0xAB, dtype=torch.uint8, device="cuda")
+    hif4.hif4_quantize(view, mode, out=out[1:38])
+    _compare_units(out[1:38].cpu().numpy(), oracle.quantize(np.ascontiguousarray(tame[:37, 64:384]), mode), "fp16 strided")
+    assert (out[0] == 0xAB).all() and (out[38] == 0xAB).all()
+    with pytest.raises(hif4.Hif4Error):
+        hif4.hif4_dequantize(out[1:38].contiguous(), dtype=torch.float16)     # FP16 is a source type only
+    # hif4_linear on FP16 activations = quantize + GEMM
+    g = torch.Generator(device="cuda"); g.manual_seed(9 + mode)
+    x16 = torch.randn(24, 512, generator=g, device="cuda").to(torch.float16)
+    w = hif4.hif4_quantize((torch.randn(96, 512, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
+    y = hif4.hif4_linear(x16, w, mode=mode)
+    assert torch.equal(y, hif4.hif4_gemm(hif4.hif4_quantize(x16, mode), w))

@@ -159,6 +159,40 @@ def test_worked_example_fp32_source():
     assert codes_of(u32)[0] == 6 and codes_of(u16)[0] == 6
 
 
+def test_worked_examples_fp16_source():
+    """FP16 source (Section II-B: "FP32 and FP16"): elements are widened to FP32 and Algorithm 1 runs in FP32
+    arithmetic.  Hand cases: the FP32 example above with FP16 storage, where x8 = fp16(0.0585) =
+    0.058502197265625: 0.0585022 * 6.4000001 = 0.374414 -> 1.49766 quarters -> code 1 (narrowing the source
+    to BF16 instead would give 0.05859375 and the tie code 2); the smallest FP16 subnormal 2^-24:
+    SF = 2^-24 / 7 = 1.1428 * 2^-27 -> E6M2 1.25 * 2^-27 = byte (21 << 2) | 1 = 0x55, REC = 0.8 * 2^27,
+    t = 6.4 with both micro-exponents -> 1.6 -> code 6 (1.5), value 1.5 * 4 * 1.25 * 2^-27 = 0.9375 * 2^-24;
+    the largest FP16 65504: SF = 9357.7 = 1.1423 * 2^13 -> byte (61 << 2) | 1 = 0xF5 (no saturation)."""
+    x = np.zeros((1, 64), dtype=np.float16)
+    x[0, 63] = -7.0
+    u = oracle.quantize(x)[0, 0]
+    assert meta_of(u) == (0xC0 | (1 << 15) | (1 << 31)) and codes_of(u)[63] == 0xF
+    x[0, 63] = 0.0
+    x[0, 0] = 1.0
+    x[0, 8] = 0.0585
+    assert float(x[0, 8]) == 0.058502197265625
+    u = oracle.quantize(x)[0, 0]
+    assert (meta_of(u) & 0xFF) == 0xB5 and codes_of(u)[8] == 1 and codes_of(u)[0] == 6
+    assert codes_of(oracle.quantize(to_bf16_bits(x.astype(np.float32)))[0, 0])[8] == 2
+    t = np.zeros((1, 64), dtype=np.float16)
+    t[0, 5] = 2.0 ** -24
+    u = oracle.quantize(t)[0, 0]
+    assert meta_of(u) == (0x55 | (1 << 8) | (1 << 17)) and codes_of(u)[5] == 6
+    assert oracle.dequantize(u.reshape(1, 1, 36))[0, 5] == 0.9375 * 2.0 ** -24
+    t[0, 5] = 65504.0
+    u = oracle.quantize(t)[0, 0]
+    assert (meta_of(u) & 0xFF) == 0xF5
+    t[0, 9] = np.nan
+    assert meta_of(oracle.quantize(t)[0, 0]) == 0xFF
+    t[0, 9] = -np.inf                                   # Inf is not NaN: top scale, the element clamps to -1.75 * 4
+    u = oracle.quantize(t)[0, 0]
+    assert (meta_of(u) & 0xFF) == 0xFE and codes_of(u)[9] == 0xF
+
+
 # ------------------------------------------------------------------ special inputs
 def test_special_inputs():
     z = np.zeros(64, dtype=np.float32)
