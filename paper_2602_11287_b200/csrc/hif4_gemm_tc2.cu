@@ -66,13 +66,66 @@ struct Gemm2Params {
   int total_tiles;
   unsigned int* error_word;
   int tma_store;        // 1: C goes out through the tensor map tmC, 0: per-thread stores
+  // Tail of the tile schedule: every pair computes `full_rounds` whole tiles; the `tail_tiles` tiles that
+  // are left (fewer than there are pairs) are cut into `slices` K ranges each, so that the last round
+  // keeps tail_tiles * slices pairs busy instead of tail_tiles.  Slice 0 of a tile stores its part to C,
+  // slice s > 0 adds its part with TMA reduce-add stores once slice s - 1 has finished the same rows
+  // (warp to warp: an epilogue warp owns 32 rows of the tile), so every element is summed in slice order.
+  int full_rounds;
+  int tail_tiles;
+  int slices;               // 1: tail tiles are not split
+  unsigned int* flags;      // [tail_tiles][slices][8]: "this epilogue warp's rows of this slice are in C" (zero at launch)
   DecodeMul mul;
 };
 
-struct PairTile { int m0; int n0; };
-__device__ __forceinline__ PairTile pair_tile(const Gemm2Params& p, int t) {
+constexpr int kMaxSlices = 4;
+constexpr int kMinSliceChunks = 4;
+
+struct WorkItem {
+  int m0, n0;           // tile origin
+  int kc0, kc1;         // K = 256 chunks [kc0, kc1)
+  int tail;             // index among the tail tiles, -1 for a whole tile
+  int slice;            // K slice of a tail tile
+};
+__device__ __forceinline__ int num_work_items(const Gemm2Params& p, int pair) {
+  return p.full_rounds + (pair < p.tail_tiles * p.slices ? 1 : 0);
+}
+__device__ __forceinline__ WorkItem work_item(const Gemm2Params& p, int pair, int num_pairs, int i) {
+  WorkItem w;
+  int t;
+  if (i < p.full_rounds) {
+    t = i * num_pairs + pair;
+    w.kc0 = 0; w.kc1 = p.num_kc; w.tail = -1; w.slice = 0;
+  } else {
+    w.tail = pair % p.tail_tiles;
+    w.slice = pair / p.tail_tiles;
+    t = p.full_rounds * num_pairs + w.tail;
+    w.kc0 = static_cast<int>(static_cast<int64_t>(w.slice) * p.num_kc / p.slices);
+    w.kc1 = static_cast<int>(static_cast<int64_t>(w.slice + 1) * p.num_kc / p.slices);
+  }
   const int mt = t / p.n_tiles;
-  return PairTile{mt * kPairM, (t - mt * p.n_tiles) * kPairN};
+  w.m0 = mt * kPairM;
+  w.n0 = (t - mt * p.n_tiles) * kPairN;
+  return w;
+}
+
+// Bounded wait until a word in global memory, written by another CTA after a __threadfence(), has reached
+// `want`.  Returns false when the budget ran out or another thread has already given up.
+__device__ __noinline__ bool wait_count(const unsigned int* counter, unsigned int want, volatile uint32_t* abort_flag) {
+  const uint64_t t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+    if (v >= want) return true;
+    __nanosleep(128);
+    if ((it & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > kWaitBudgetNs) {
+        *abort_flag = 1u;
+        return false;
+      }
+    }
+  }
 }
 
 // Decodes the two units held in raw words W[0..8] and W[9..17] into decoded stages 2h and 2h+1.  Returns
@@ -116,6 +169,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+  const int n_items = num_work_items(p, pair);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kRawStages; ++s) {
@@ -150,15 +204,15 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (lane == 0) {
       uint32_t n = 0;
       bool ok = true;
-      for (int t = pair; t < p.total_tiles && ok; t += num_pairs) {
-        const PairTile tc = pair_tile(p, t);
-        for (int kc = 0; kc < p.num_kc; ++kc, ++n) {
+      for (int i = 0; i < n_items && ok; ++i) {
+        const WorkItem w = work_item(p, pair, num_pairs, i);
+        for (int kc = w.kc0; kc < w.kc1; ++kc, ++n) {
           const uint32_t s = n & 1u, ph = (n >> 1) & 1u;
           if (!(ok = mbar_wait(raw_empty + 8 * s, ph ^ 1u, abort_flag, 128))) break;
           mbar_expect_tx(raw_full + 8 * s, kRawStageBytes);
           const uint32_t dst = raw_base + s * kRawStageBytes;
-          tma_load_2d(dst, &tmA, kc * kRawRowBytes, tc.m0 + static_cast<int>(rank) * kRows, raw_full + 8 * s);
-          tma_load_2d(dst + kRawHalfBytes, &tmB, kc * kRawRowBytes, tc.n0 + static_cast<int>(rank) * kRows,
+          tma_load_2d(dst, &tmA, kc * kRawRowBytes, w.m0 + static_cast<int>(rank) * kRows, raw_full + 8 * s);
+          tma_load_2d(dst + kRawHalfBytes, &tmB, kc * kRawRowBytes, w.n0 + static_cast<int>(rank) * kRows,
                       raw_full + 8 * s);
         }
       }
@@ -168,12 +222,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (rank == 0 && lane == 0) {
       uint32_t n = 0, tcount = 0;
       bool ok = true;
-      for (int t = pair; t < p.total_tiles && ok; t += num_pairs, ++tcount) {
+      for (int it = 0; it < n_items && ok; ++it, ++tcount) {
+        const WorkItem w = work_item(p, pair, num_pairs, it);
         const uint32_t acc = tcount & 1u, aph = (tcount >> 1) & 1u;
         if (!(ok = mbar_wait_cluster(tmem_empty + 8 * acc, aph ^ 1u, abort_flag))) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * kPairN;
-        for (int kc = 0; kc < p.num_kc && ok; ++kc, ++n) {
+        for (int kc = w.kc0; kc < w.kc1 && ok; ++kc, ++n) {
           // The two halves of the decode threads fill stages (0, 1) and (2, 3) side by side, so stages
           // 0 and 2 are ready first: the K blocks of a chunk are consumed in the order 0, 2, 1, 3.
 #pragma unroll
@@ -185,7 +240,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const uint64_t bdesc = make_desc(dec_base + u * kDecStageBytes + kDecHalfBytes);
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-              tc2_mma(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, kInstrDesc2, (kc | i | kk) != 0 ? 1u : 0u);
+              tc2_mma(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, kInstrDesc2, ((kc - w.kc0) | i | kk) != 0 ? 1u : 0u);
             tc2_commit_both(dec_empty + 8 * u);       // both CTAs may overwrite the stage once these MMAs have read it
           }
         }
@@ -205,17 +260,22 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const uint32_t my_row = slab0 + static_cast<uint32_t>(lane) * 64u;
       const uint32_t sw = (static_cast<uint32_t>(lane) >> 1) & 3u;
       uint32_t slabs = 0;
-      for (int t = pair; t < p.total_tiles; t += num_pairs, ++tcount) {
-        const PairTile tc = pair_tile(p, t);
+      for (int it = 0; it < n_items; ++it, ++tcount) {
+        const WorkItem w = work_item(p, pair, num_pairs, it);
         const uint32_t acc = tcount & 1u, aph = (tcount >> 1) & 1u;
         if (!__all_sync(0xFFFFFFFFu, mbar_wait(tmem_full + 8 * acc, aph, abort_flag, 256))) break;
         tc_fence_after();
-        const int row0 = tc.m0 + static_cast<int>(rank) * kRows + q * 32;
+        // K-sliced tail tile: slice 0 stores, slice s > 0 adds once the same warp of slice s - 1 is done
+        const bool sliced = w.tail >= 0 && p.slices > 1;
+        const bool adds = sliced && w.slice > 0;
+        unsigned int* my_flag = sliced ? p.flags + (static_cast<size_t>(w.tail) * p.slices + w.slice) * 8 + rank * 4 + q : nullptr;
+        if (adds && !__all_sync(0xFFFFFFFFu, wait_count(my_flag - 8, 1u, abort_flag))) break;
+        const int row0 = w.m0 + static_cast<int>(rank) * kRows + q * 32;
 #pragma unroll 1
         for (int c = 0; c < kPairN / kEpiCols; ++c) {
           // slabs that lie entirely outside C are neither read nor staged: the two staging buffers
           // alternate over the slabs that are stored, which is what the wait below counts on
-          const bool stored = row0 < p.M && tc.n0 + c * kEpiCols < p.N;            // same for the whole warp
+          const bool stored = row0 < p.M && w.n0 + c * kEpiCols < p.N;             // same for the whole warp
           uint32_t r[16];
           if (stored) {
             tc_ld16(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kPairN + c * kEpiCols, r);
@@ -236,29 +296,35 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           fence_proxy_async_smem();                  // generic-proxy writes -> visible to the TMA store
           __syncwarp();
           if (lane == 0) {
-            tma_store_2d(&tmC, tc.n0 + c * kEpiCols, row0, slab0 + buf);
+            if (adds) tma_reduce_add_2d(&tmC, w.n0 + c * kEpiCols, row0, slab0 + buf);
+            else tma_store_2d(&tmC, w.n0 + c * kEpiCols, row0, slab0 + buf);
             bulk_commit();
           }
           ++slabs;
+        }
+        if (sliced && w.slice + 1 < p.slices && lane == 0) {      // the next slice may add to these rows now
+          bulk_wait_all();
+          __threadfence();
+          asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(my_flag), "r"(1u) : "memory");
         }
       }
       if (lane == 0) bulk_wait_all();                // shared memory stays valid until the last store has read it
     } else {
       const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15u) == 0) && (p.ldc % 4 == 0);
-      for (int t = pair; t < p.total_tiles; t += num_pairs, ++tcount) {
-        const PairTile tc = pair_tile(p, t);
+      for (int it = 0; it < n_items; ++it, ++tcount) {         // (tail tiles are never K-sliced on this path)
+        const WorkItem w = work_item(p, pair, num_pairs, it);
         const uint32_t acc = tcount & 1u, aph = (tcount >> 1) & 1u;
         if (!__all_sync(0xFFFFFFFFu, mbar_wait(tmem_full + 8 * acc, aph, abort_flag, 256))) break;
         tc_fence_after();
-        const int64_t row = static_cast<int64_t>(tc.m0) + rank * kRows + q * 32 + lane;
+        const int64_t row = static_cast<int64_t>(w.m0) + rank * kRows + q * 32 + lane;
         const bool row_ok = row < p.M;
-        float* crow = p.C + row * p.ldc + tc.n0;
+        float* crow = p.C + row * p.ldc + w.n0;
 #pragma unroll 1
         for (int c = 0; c < kPairN / 32; ++c) {
           uint32_t r[32];
           tc_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kPairN + c * 32, r);
           tc_wait_ld();
-          const int64_t col0 = static_cast<int64_t>(tc.n0) + c * 32;
+          const int64_t col0 = static_cast<int64_t>(w.n0) + c * 32;
           if (row_ok && col0 < p.N) {
             if (vec_ok && col0 + 32 <= p.N) {
 #pragma unroll
@@ -292,8 +358,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t dec_full0_leader = mapa(dec_full, 0) + 16 * h;
     uint32_t n = 0;
     bool ok = true;
-    for (int t = pair; t < p.total_tiles && ok; t += num_pairs) {
-      for (int kc = 0; kc < p.num_kc && ok; ++kc, ++n) {
+    for (int i = 0; i < n_items && ok; ++i) {
+      const WorkItem w = work_item(p, pair, num_pairs, i);
+      for (int kc = w.kc0; kc < w.kc1 && ok; ++kc, ++n) {
         const uint32_t s = n & 1u, ph = (n >> 1) & 1u;
         if (!(ok = __all_sync(0xFFFFFFFFu, mbar_wait(raw_full + 8 * s, ph, abort_flag)))) break;
         uint32_t L[20];
@@ -348,13 +415,47 @@ bool make_c_map(CUtensorMap* map, float* C, int64_t M, int64_t N, int64_t ldc) {
 
 }  // namespace
 
+// Tile schedule of the dense pair kernel for this shape on this device (see Gemm2Params).
+struct Tc2Plan {
+  int pairs, full_rounds, tail_tiles, slices;
+  size_t flag_bytes, bytes;          // workspace: the slices' completion words
+};
+static Tc2Plan tc2_plan(int64_t M, int64_t N, int64_t K) {
+  Tc2Plan pl{};
+  const int64_t tiles = ceil_div64(M, kPairM) * ceil_div64(N, kPairN);
+  const int64_t max_pairs = sm_count() / 2;
+  pl.pairs = static_cast<int>(tiles < max_pairs ? tiles : max_pairs);
+  pl.slices = 1;
+  if (pl.pairs <= 0 || tiles > 0x7FFFFFFFll) return pl;
+  pl.full_rounds = static_cast<int>(tiles / pl.pairs);
+  pl.tail_tiles = static_cast<int>(tiles % pl.pairs);
+  if (pl.tail_tiles > 0) {
+    // Slice s starts its epilogue when slice s - 1 has finished its own, so every slice adds an epilogue's
+    // length to the tile: it has to be at least kMinSliceChunks K = 256 chunks long to win that back.
+    int64_t s = pl.pairs / pl.tail_tiles;
+    if (s > kMaxSlices) s = kMaxSlices;
+    if (s > K / (256 * kMinSliceChunks)) s = K / (256 * kMinSliceChunks);
+    if (s >= 2) pl.slices = static_cast<int>(s);
+  }
+  if (pl.slices > 1) {
+    pl.flag_bytes = (static_cast<size_t>(pl.tail_tiles) * pl.slices * 8 * sizeof(unsigned int) + 255) / 256 * 256;
+    pl.bytes = pl.flag_bytes;
+  }
+  return pl;
+}
+
+size_t gemm_tc2_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  if (M <= 0 || N <= 0 || K <= 0 || K % 256 != 0) return 0;
+  return tc2_plan(M, N, K).bytes;
+}
+
 bool gemm_tc2_supported(const void* A, const void* B, int64_t M, int64_t N, int64_t K) {
   if (!gemm_tc_supported(A, B, M, N, N, K)) return false;
   return M < (1ll << 31) - kPairM && N < (1ll << 31) - kPairN && sm_count() >= 2;
 }
 
 hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,
-                            cudaStream_t st) {
+                            void* workspace, size_t workspace_bytes, cudaStream_t st) {
   static uint64_t smem_opt_in = 0;
   if (!ensure_dynamic_smem(gemm_tc2_kernel, kSmemBytes, smem_opt_in)) return HIF4_ERR_CUDA;
   CUtensorMap tmA, tmB;
@@ -372,8 +473,16 @@ hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, i
   p.mul = make_decode_mul();
   CUtensorMap tmC = tmA;                              // placeholder when the store path is not used
   p.tma_store = ((reinterpret_cast<uintptr_t>(C) & 15u) == 0 && ldc % 4 == 0 && make_c_map(&tmC, C, M, N, ldc)) ? 1 : 0;
-  const int pairs = static_cast<int>(tiles < sm_count() / 2 ? tiles : sm_count() / 2);
-  gemm_tc2_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tmA, tmB, tmC, p);
+  const Tc2Plan pl = tc2_plan(M, N, K);
+  p.full_rounds = pl.full_rounds;
+  p.tail_tiles = pl.tail_tiles;
+  p.slices = p.tma_store ? pl.slices : 1;             // the plain-store epilogue cannot add to C
+  if (p.slices > 1) {
+    if (!workspace || workspace_bytes < pl.bytes) return HIF4_ERR_WORKSPACE;
+    p.flags = static_cast<unsigned int*>(workspace);
+    if (cudaMemsetAsync(p.flags, 0, pl.flag_bytes, st) != cudaSuccess) return HIF4_ERR_CUDA;
+  }
+  gemm_tc2_kernel<<<2 * pl.pairs, kThreads, kSmemBytes, st>>>(tmA, tmB, tmC, p);
   note_launch();
   return launch_status();
 }

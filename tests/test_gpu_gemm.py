@@ -222,6 +222,33 @@ def test_cta_pair_kernel_few_columns_in_the_last_tile_repeated(hif4):
     assert hif4.hif4_last_device_status() == 0
 
 
+@pytest.mark.parametrize("M,N,K", [(2560, 2048, 16384), (2500, 2000, 8192), (19 * 256, 4 * 256 + 8, 8192), (2560, 2048, 2048)])
+def test_cta_pair_kernel_k_sliced_last_round(hif4, M, N, K):
+    """More tiles than CTA pairs with a partial last round: its tiles are cut into K slices that are added to
+    C in slice order (80 tiles on 74 pairs -> 6 tail tiles x 4 or 2 slices; 95 tiles -> 21 tail tiles x 3)."""
+    assert hif4.hif4_gemm_workspace(M, N, K) > 0, "the K-sliced round needs its completion words"
+    g = torch.Generator(device="cuda"); g.manual_seed(M + N + K)
+    a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
+    b = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
+    out = torch.full((M + 2, N + 4), -3.0, dtype=torch.float32, device="cuda")
+    C = check_sampled(hif4, a, b, f"k-sliced {M}x{N}x{K}", n=1500, seed=K, C=hif4.hif4_gemm(a, b, out=out[1:M + 1, :N]))
+    assert (out[0] == -3.0).all() and (out[M + 1] == -3.0).all() and (out[:, N:] == -3.0).all()
+    # every entry of the tail tiles against the kernel that never slices (different FP32 summation order)
+    hif4.hif4_set_gemm_path(2)
+    try:
+        C1 = hif4.hif4_gemm(a, b)
+    finally:
+        hif4.hif4_set_gemm_path(0)
+    scale = (C1.abs().max() + 1e-30).item()
+    assert (C.contiguous() - C1).abs().max().item() <= 1e-5 * scale * K
+    for _ in range(3):
+        assert torch.equal(hif4.hif4_gemm(a, b), C.contiguous()), "K-sliced tiles are not reproducible"
+    with pytest.raises(hif4.Hif4Error) as ei:
+        hif4.hif4_gemm(a, b, workspace=torch.empty(64, dtype=torch.uint8, device="cuda"))
+    assert ei.value.code == 5
+    assert hif4.hif4_last_device_status() == 0
+
+
 def test_tensor_core_kernel_c_rows_not_16_byte_aligned(tc_path):
     """ldc odd and a base that is only 4-byte aligned: the kernels fall back from vector / TMA stores."""
     hif4 = tc_path
