@@ -79,7 +79,6 @@ struct Gemm2Params {
 };
 
 constexpr int kMaxSlices = 4;
-constexpr int kMinSliceChunks = 4;
 
 struct WorkItem {
   int m0, n0;           // tile origin
@@ -429,13 +428,22 @@ static Tc2Plan tc2_plan(int64_t M, int64_t N, int64_t K) {
   if (pl.pairs <= 0 || tiles > 0x7FFFFFFFll) return pl;
   pl.full_rounds = static_cast<int>(tiles / pl.pairs);
   pl.tail_tiles = static_cast<int>(tiles % pl.pairs);
+  if (tiles < max_pairs) {            // a single, partial round: all its tiles are "tail" tiles
+    pl.full_rounds = 0;
+    pl.tail_tiles = static_cast<int>(tiles);
+  }
   if (pl.tail_tiles > 0) {
-    // Slice s starts its epilogue when slice s - 1 has finished its own, so every slice adds an epilogue's
-    // length to the tile: it has to be at least kMinSliceChunks K = 256 chunks long to win that back.
-    int64_t s = pl.pairs / pl.tail_tiles;
-    if (s > kMaxSlices) s = kMaxSlices;
-    if (s > K / (256 * kMinSliceChunks)) s = K / (256 * kMinSliceChunks);
-    if (s >= 2) pl.slices = static_cast<int>(s);
+    // Slice s starts its epilogue when slice s - 1 has finished its own, which adds about the time of
+    // 3.5 K = 256 chunks per extra slice (measured): take the slice count with the shortest critical path.
+    int64_t s_max = max_pairs / pl.tail_tiles;
+    if (s_max > kMaxSlices) s_max = kMaxSlices;
+    const int64_t chunks = K / 256;
+    int64_t best = 1, best_cost = 2 * chunks;
+    for (int64_t s = 2; s <= s_max; ++s) {
+      const int64_t cost = 2 * ceil_div64(chunks, s) + 7 * (s - 1);       // in half chunks
+      if (cost < best_cost) { best = s; best_cost = cost; }
+    }
+    pl.slices = static_cast<int>(best);
   }
   if (pl.slices > 1) {
     pl.flag_bytes = (static_cast<size_t>(pl.tail_tiles) * pl.slices * 8 * sizeof(unsigned int) + 255) / 256 * 256;
@@ -482,7 +490,8 @@ hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, i
     p.flags = static_cast<unsigned int*>(workspace);
     if (cudaMemsetAsync(p.flags, 0, pl.flag_bytes, st) != cudaSuccess) return HIF4_ERR_CUDA;
   }
-  gemm_tc2_kernel<<<2 * pl.pairs, kThreads, kSmemBytes, st>>>(tmA, tmB, tmC, p);
+  const int pairs = p.full_rounds == 0 ? p.tail_tiles * p.slices : pl.pairs;      // a single round: one pair per slice
+  gemm_tc2_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tmA, tmB, tmC, p);
   note_launch();
   return launch_status();
 }
