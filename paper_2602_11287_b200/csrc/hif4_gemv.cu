@@ -139,14 +139,12 @@ __device__ __forceinline__ UnitPrep prepare_unit(uint32_t meta, uint32_t lut) {
 __device__ __forceinline__ void decode_word(const UnitPrep& u, int j, uint32_t wj, const DecodeMul& k, uint32_t (&r)[4]) {
   const uint32_t f = ((u.sum >> (2 * j)) * k.m128) & 0x01800180u;    // field j at the exponent's low bits
   const uint32_t Sa = f * k.one + u.base2;                          // (S_lo, S_hi), S = E6M2 * 2^(e8 + e16 - 2)
-  const uint32_t Sb = Sa - 0x02000200u;                             // S / 16
-  const uint32_t Oa = Sa * k.one + 0x83808380u;                     // -128 S
-  const uint32_t Ob = Sa * k.one + 0x81808180u;                     // -8 S
-  const uint32_t wh = wj >> 8;
-  r[0] = fma_bf16x2((wj & 0x00070007u) | u.or_k, Sa, Oa) ^ ((wj * k.m4096) & 0x80008000u);
-  r[1] = fma_bf16x2((wj & 0x00700070u) | u.or_k, Sb, Ob) ^ ((wj * k.m256) & 0x80008000u);
-  r[2] = fma_bf16x2((wh & 0x00070007u) | u.or_k, Sa, Oa) ^ ((wj * k.m16) & 0x80008000u);
-  r[3] = fma_bf16x2((wh & 0x00700070u) | u.or_k, Sb, Ob) ^ (wj & 0x80008000u);
+  const uint32_t Oa = mul_bf16x2(Sa, 0xC308C308u);                  // -136 S
+  const uint32_t uj = offset_nibbles(wj, k);                        // nibbles 8 + value: no separate sign step
+  r[0] = fma_bf16x2((uj & 0x000F000Fu) | u.or_k, Sa, Oa);           // (128 + u) S - 136 S
+  r[1] = fma_bf16x2(((uj >> 4) & 0x000F000Fu) | u.or_k, Sa, Oa);
+  r[2] = fma_bf16x2(((uj >> 8) & 0x000F000Fu) | u.or_k, Sa, Oa);
+  r[3] = fma_bf16x2(((uj >> 12) & 0x000F000Fu) | u.or_k, Sa, Oa);
 }
 
 // A parity wait cannot tell a barrier that is one phase behind from one that is done, so a consumer

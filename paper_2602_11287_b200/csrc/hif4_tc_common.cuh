@@ -104,6 +104,11 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
 __device__ __forceinline__ uint32_t fma_bf16x2(uint32_t a, uint32_t b, uint32_t c) {
   uint32_t d;
   asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
@@ -154,10 +159,18 @@ __device__ __forceinline__ void decode_unit_to_row(uint32_t meta, const uint32_t
 // additions onto that pipe by writing them as multiply-adds with multipliers that the compiler cannot
 // see (kernel parameters), takes the sum of the micro-exponents of all eight level-2 groups at once
 // (two-bit fields), and uses store addresses that are computed once per thread.
-struct DecodeMul {            // runtime-valued on purpose: 1, 2, 8, 16, 32, 128, 256, 4096
-  uint32_t one, m2, m8, m16, m32, m128, m256, m4096;
+struct DecodeMul {            // runtime-valued on purpose: 1, 2, 7, 8, 32, 128
+  uint32_t one, m2, m7, m8, m32, m128;
 };
-inline DecodeMul make_decode_mul() { return DecodeMul{1u, 2u, 8u, 16u, 32u, 128u, 256u, 4096u}; }
+inline DecodeMul make_decode_mul() { return DecodeMul{1u, 2u, 7u, 8u, 32u, 128u}; }
+
+// The eight sign-magnitude nibbles (s, m) of a code word -> offset nibbles u = 8 + value (1..15), all at
+// once: u = c ^ 8 for s = 0 and 16 - c for s = 1, i.e. (c ^ (8 | 7s)) + s with no carry out of a nibble.
+// An element then decodes as (128 + u) * S - 136 * S with no separate sign step (-0 decodes as +0).
+__device__ __forceinline__ uint32_t offset_nibbles(uint32_t w, const DecodeMul& k) {
+  const uint32_t s1 = (w & 0x88888888u) >> 3;                       // 1 in every negative nibble
+  return (w ^ (s1 * k.m7 | 0x88888888u)) + s1 * k.one;
+}
 
 // 256-entry table in shared memory: bit i of the index spread to bit 2i, replicated in both halves.
 __device__ __forceinline__ uint32_t spread_e8_entry(uint32_t x) {
@@ -194,14 +207,12 @@ __device__ __forceinline__ void decode_unit_balanced(uint32_t meta, const uint32
   for (int j = 0; j < 8; ++j) {
     const uint32_t f = ((j < 4 ? sum : sumh) * mul[j & 3]) & 0x01800180u;       // field j at the exponent's low bits
     const uint32_t Sa = f * k.one + base2;                            // (S_lo, S_hi), S = E6M2 * 2^(e8 + e16 - 2)
-    const uint32_t Sb = Sa - 0x02000200u;                             // S / 16
-    const uint32_t Oa = Sa * k.one + 0x83808380u;                     // -128 S
-    const uint32_t Ob = Sa * k.one + 0x81808180u;                     // -8 S
-    const uint32_t wj = w[j], wh = wj >> 8;
-    const uint32_t r0 = fma_bf16x2((wj & 0x00070007u) | 0x43004300u, Sa, Oa) ^ ((wj * k.m4096) & 0x80008000u);  // elements 0, 4
-    const uint32_t r1 = fma_bf16x2((wj & 0x00700070u) | 0x43004300u, Sb, Ob) ^ ((wj * k.m256) & 0x80008000u);   // elements 1, 5
-    const uint32_t r2 = fma_bf16x2((wh & 0x00070007u) | 0x43004300u, Sa, Oa) ^ ((wj * k.m16) & 0x80008000u);    // elements 2, 6
-    const uint32_t r3 = fma_bf16x2((wh & 0x00700070u) | 0x43004300u, Sb, Ob) ^ (wj & 0x80008000u);              // elements 3, 7
+    const uint32_t Oa = mul_bf16x2(Sa, 0xC308C308u);                  // -136 S
+    const uint32_t uj = offset_nibbles(w[j], k);
+    const uint32_t r0 = fma_bf16x2((uj & 0x000F000Fu) | 0x43004300u, Sa, Oa);           // elements 0, 4: (128 + u) S - 136 S
+    const uint32_t r1 = fma_bf16x2(((uj >> 4) & 0x000F000Fu) | 0x43004300u, Sa, Oa);    // elements 1, 5
+    const uint32_t r2 = fma_bf16x2(((uj >> 8) & 0x000F000Fu) | 0x43004300u, Sa, Oa);    // elements 2, 6
+    const uint32_t r3 = fma_bf16x2(((uj >> 12) & 0x000F000Fu) | 0x43004300u, Sa, Oa);   // elements 3, 7
     sts128(chunk_addr[j] + stage_off, r0, r1, r2, r3);
   }
 }
