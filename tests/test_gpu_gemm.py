@@ -159,6 +159,36 @@ def test_grouped_gemm_moe_routing_sampled(hif4):
     assert np.all(err <= TOL * refabs + 1e-300)
 
 
+def test_grouped_gemm_many_small_groups_wide_n(hif4):
+    """Many experts with few rows and a wide N (8192 rows, 140 groups of 1..130 rows + empty ones, N = 8192 + 40:
+    33 weight tiles per token tile, the last one ragged): thousands of small work units per launch.  Compared
+    entry by entry with the single-CTA kernel, and sampled against the oracle."""
+    rng = np.random.default_rng(77)
+    sizes = list(rng.integers(1, 131, 140))
+    sizes[5] = 0; sizes[60] = 0
+    sizes[-1] += 8192 - sum(sizes) if sum(sizes) < 8192 else 0
+    G, K, N = len(sizes), 256, 8192 + 40
+    off = torch.tensor(np.concatenate([[0], np.cumsum(sizes)]), dtype=torch.int64, device="cuda")
+    total = int(off[-1])
+    g = torch.Generator(device="cuda"); g.manual_seed(78)
+    a = hif4.hif4_quantize(torch.randn(total, K, generator=g, device="cuda").to(torch.bfloat16))
+    b = hif4.hif4_quantize((torch.randn(G * N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16)).view(G, N, K // 64, 36)
+    out = hif4.hif4_grouped_gemm(a, b, off)
+    assert torch.equal(out, hif4.hif4_grouped_gemm(a, b, off)), "two runs differ"
+    hif4.hif4_set_gemm_path(2)
+    try:
+        ref1 = hif4.hif4_grouped_gemm(a, b, off)
+    finally:
+        hif4.hif4_set_gemm_path(0)
+    assert (out - ref1).abs().max().item() <= 1e-5 * K * ref1.abs().max().item()
+    off_h = off.cpu().numpy()
+    for gsel in (0, 7, 60, 61, G - 1):
+        lo, hi = int(off_h[gsel]), int(off_h[gsel + 1])
+        if hi > lo:
+            check_sampled(hif4, a[lo:hi], b[gsel], f"group {gsel}", n=400, seed=gsel, C=out[lo:hi])
+    assert hif4.hif4_last_device_status() == 0
+
+
 # ------------------------------------------------------------------ tensor-core (tcgen05) kernel
 @pytest.fixture(params=[2, 3], ids=["one_cta", "cta_pair"])
 def tc_path(hif4, request):
