@@ -28,7 +28,9 @@ constexpr int kBlockRows = 8;                        // granule of the row parti
 constexpr int kBlockBytes = kBlockRows * kRawRowBytes;   // 1152 = 9 * 128
 constexpr int kMaxBlocks = 16;                       // 8-row blocks per CTA (TMA box of up to 128 rows)
 constexpr int kMaxStages = 16;
-constexpr int kGemvWarps = 24;                       // consumer warps per CTA
+// consumer warps per CTA: 31 when a CTA owns many rows (five row pairs or more share them evenly and hide
+// more latency), 24 otherwise (fewer warps wait on the same few chunks)
+constexpr int kGemvWarpsMany = 31, kGemvWarpsFew = 24;
 constexpr int kRingBudget = 176 * 1024;              // bytes of shared memory given to the ring of stages
 
 struct GemvParams {
@@ -167,7 +169,7 @@ __device__ __forceinline__ bool wait_announced(const volatile int* slot, int kc,
 }
 
 // Shared memory: [spread table 1 KB][partial sums][barriers, abort word, announced chunks: 384 B][ring of stages, 128-byte aligned]
-template <int kTokTiles>
+template <int kTokTiles, int kGemvWarps>
 __global__ void __launch_bounds__((kGemvWarps + 1) * 32, 1)
 gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__ CUtensorMap tm_short, const GemvParams p) {
   constexpr int kTokBytes = kTokTiles * kTileChunkBytes;
@@ -313,7 +315,7 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
   }
 }
 
-template <int kTokTiles>
+template <int kTokTiles, int kGemvWarps>
 hif4_status launch_gemv_t(const void* B, int64_t upr, GemvParams p, cudaStream_t st) {
   constexpr int kTokBytes = kTokTiles * kTileChunkBytes;
   constexpr int kFixed = 128 + 1024 + kGemvWarps * 32 * 4 * kTokTiles * 4 + 384;
@@ -329,7 +331,7 @@ hif4_status launch_gemv_t(const void* B, int64_t upr, GemvParams p, cudaStream_t
   if (p.stages > p.num_kc) p.stages = p.num_kc;
   const int smem = kFixed + p.stages * stage_bytes;
   static uint64_t smem_opt_in = 0;
-  if (!ensure_dynamic_smem(gemv_kernel<kTokTiles>, kFixed + kRingBudget, smem_opt_in)) return HIF4_ERR_CUDA;
+  if (!ensure_dynamic_smem(gemv_kernel<kTokTiles, kGemvWarps>, kFixed + kRingBudget, smem_opt_in)) return HIF4_ERR_CUDA;
   CUtensorMap tm_full, tm_short;
   if (!make_unit_map(&tm_full, B, p.N, upr, p.max_blocks * kBlockRows)) return HIF4_ERR_CUDA;
   if (!make_unit_map(&tm_short, B, p.N, upr, (p.max_blocks > 1 ? p.max_blocks - 1 : 1) * kBlockRows)) return HIF4_ERR_CUDA;
@@ -343,7 +345,7 @@ hif4_status launch_gemv_t(const void* B, int64_t upr, GemvParams p, cudaStream_t
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, gemv_kernel<kTokTiles>, tm_full, tm_short, p) != cudaSuccess) {
+  if (cudaLaunchKernelEx(&cfg, gemv_kernel<kTokTiles, kGemvWarps>, tm_full, tm_short, p) != cudaSuccess) {
     (void)cudaGetLastError();
     return HIF4_ERR_CUDA;
   }
@@ -381,7 +383,13 @@ hif4_status launch_gemv(const void* A, const void* B, float* C, int64_t M, int64
   gemv_prepare_tokens_kernel<<<static_cast<unsigned>(ceil_div64(prep, 128)), 128, 0, st>>>(p.A, p.M, m_pad, upr, p.tokens);
   note_launch();
   if (cudaGetLastError() != cudaSuccess) return HIF4_ERR_CUDA;
-  return m_pad == 8 ? launch_gemv_t<1>(B, upr, p, st) : launch_gemv_t<2>(B, upr, p, st);
+  // blocks of the largest CTA (same arithmetic as launch_gemv_t): nine or more are five row pairs or more
+  const int64_t sms = sm_count();
+  const int64_t rounds = ceil_div64(p.num_blocks, sms * kMaxBlocks);
+  const int64_t grid = p.num_blocks < sms * rounds ? p.num_blocks : sms * rounds;
+  const bool many = ceil_div64(p.num_blocks, grid) >= 9;
+  if (m_pad == 8) return many ? launch_gemv_t<1, kGemvWarpsMany>(B, upr, p, st) : launch_gemv_t<1, kGemvWarpsFew>(B, upr, p, st);
+  return many ? launch_gemv_t<2, kGemvWarpsMany>(B, upr, p, st) : launch_gemv_t<2, kGemvWarpsFew>(B, upr, p, st);
 }
 
 }  // namespace hif4
