@@ -106,7 +106,8 @@ hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size_t* bytes);
  *              aligned rows (base % 16 == 0 and ldc % 4 == 0) allow vector stores.  Overwritten
  *              inside [M, N] (no alpha/beta); padding beyond N is untouched.
  *   workspace  device scratch of at least hif4_gemm_workspace bytes, 256-byte aligned, contents
- *              undefined on entry and exit; may be NULL when 0 bytes are needed.
+ *              undefined on entry and exit; may be NULL when 0 bytes are needed.  Calls that may run
+ *              at the same time (different streams) need workspaces of their own.
  * K must be a multiple of 64.  M == 0 or N == 0 is a no-op; K == 0 zero-fills C.
  * Units whose E6M2 byte is NaN make every C entry they touch NaN.  */
 hif4_status hif4_gemm(const void* A_units, const void* B_units, float* C, int64_t M, int64_t N,
