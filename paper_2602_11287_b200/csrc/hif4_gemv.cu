@@ -17,6 +17,7 @@
 // Results are deterministic (no atomics).  Every mbarrier wait is bounded.
 #include "hif4_common.cuh"
 #include "hif4_gemm_internal.cuh"
+#include "hif4_quantize_device.cuh"
 #include "hif4_tc_common.cuh"
 
 namespace hif4 {
@@ -118,6 +119,47 @@ gemv_prepare_tokens_kernel(const uint32_t* __restrict__ A, int M, int m_pad, int
     decode_two_words(meta, W, __ldg(unit + 1 + W), __ldg(unit + 2 + W), r);
     *reinterpret_cast<uint4*>(dst + W * kTokChunkBytes) = make_uint4(r[0], r[1], r[2], r[3]);
     *reinterpret_cast<uint4*>(dst + (W + 1) * kTokChunkBytes) = make_uint4(r[4], r[5], r[6], r[7]);
+  }
+}
+
+// The same preparation straight from BF16 activations: Algorithm 1 (the streaming quantizer's own code, two
+// lanes per unit) followed by Eq. 2 of the unit just encoded, without the packed units ever going to memory.
+// Used by the one-call linear layer for M <= 16; the tokens written are bit-identical to quantizing first.
+template <bool kRHA>
+__global__ void __launch_bounds__(128)
+gemv_quantize_tokens_kernel(const uint16_t* __restrict__ X, int64_t ld_x, int M, int m_pad, int64_t upr,
+                            uint8_t* __restrict__ tokens) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;     // ((token n, unit U), lane l)
+  const int l = static_cast<int>(idx & 1);
+  const int64_t pair = idx >> 1;
+  const bool in_range = pair < static_cast<int64_t>(m_pad) * upr;      // same for both lanes of a pair
+  const int n = in_range ? static_cast<int>(pair / upr) : 0;
+  const int64_t U = in_range ? pair - static_cast<int64_t>(n) * upr : 0;
+  uint4 v[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) v[c] = make_uint4(0u, 0u, 0u, 0u);
+  if (in_range && n < M) {
+    const uint4* src = reinterpret_cast<const uint4*>(X + static_cast<int64_t>(n) * ld_x + U * kUnitElems) + l;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) v[c] = __ldg(src + 2 * c);
+  }
+  uint32_t codes[4], meta;
+  encode_unit_bf16_pair<kRHA>(v, l, codes, meta);        // every lane of the warp takes part (pair-wise exchange)
+  if (!in_range) return;
+  const int tiles = m_pad >> 3;
+  uint8_t* dst = tokens + (((U >> 2) * tiles + (n >> 3)) * 8) * kTokChunkBytes + ((n & 7) * 4 + (U & 3)) * 16;
+  const uint32_t byte = meta & 0xFFu;
+  const uint32_t base2 = byte * 0x00200020u + 0x26802680u;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const int W = l + 2 * c;                             // this lane's code words
+    uint32_t r[4] = {0u, 0u, 0u, 0u};
+    if (n < M) {
+      if (byte == 0xFFu) r[0] = r[1] = r[2] = r[3] = 0x7FC07FC0u;
+      else decode_word_regs(meta, base2, W, codes[c], r);
+    }
+    *reinterpret_cast<uint4*>(dst + W * kTokChunkBytes) = make_uint4(r[0], r[1], r[2], r[3]);
   }
 }
 
@@ -365,24 +407,20 @@ size_t gemv_workspace_bytes(int64_t M, int64_t K) {
   return static_cast<size_t>(m_pad * K * 2);
 }
 
-hif4_status launch_gemv(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,
-                        void* workspace, cudaStream_t st) {
-  GemvParams p{};
-  p.A = static_cast<const uint32_t*>(A);
+namespace {
+// Fills the launch parameters both entry points share; returns false when N is out of range.
+bool gemv_params(GemvParams& p, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc, void* workspace) {
   p.tokens = static_cast<uint8_t*>(workspace);
   p.C = C; p.ldc = ldc; p.M = static_cast<int>(M); p.N = N;
   p.num_kc = static_cast<int>(K / 256);
-  if (ceil_div64(N, kBlockRows) > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
+  if (ceil_div64(N, kBlockRows) > 0x7FFFFFFFll) return false;
   p.num_blocks = static_cast<int>(ceil_div64(N, kBlockRows));
   p.mul = make_decode_mul();
   p.error_word = device_error_word();
-  if (!p.error_word) return HIF4_ERR_CUDA;
-  const int m_pad = M <= 8 ? 8 : 16;
-  const int64_t upr = K / kUnitElems;
-  const int64_t prep = static_cast<int64_t>(m_pad) * upr;
-  gemv_prepare_tokens_kernel<<<static_cast<unsigned>(ceil_div64(prep, 128)), 128, 0, st>>>(p.A, p.M, m_pad, upr, p.tokens);
-  note_launch();
-  if (cudaGetLastError() != cudaSuccess) return HIF4_ERR_CUDA;
+  return true;
+}
+// The streaming kernel on tokens that the preceding launch in `st` has prepared.
+hif4_status launch_gemv_stream(const void* B, const GemvParams& p, int m_pad, int64_t upr, cudaStream_t st) {
   // blocks of the largest CTA (same arithmetic as launch_gemv_t): nine or more are five row pairs or more
   const int64_t sms = sm_count();
   const int64_t rounds = ceil_div64(p.num_blocks, sms * kMaxBlocks);
@@ -390,6 +428,44 @@ hif4_status launch_gemv(const void* A, const void* B, float* C, int64_t M, int64
   const bool many = ceil_div64(p.num_blocks, grid) >= 9;
   if (m_pad == 8) return many ? launch_gemv_t<1, kGemvWarpsMany>(B, upr, p, st) : launch_gemv_t<1, kGemvWarpsFew>(B, upr, p, st);
   return many ? launch_gemv_t<2, kGemvWarpsMany>(B, upr, p, st) : launch_gemv_t<2, kGemvWarpsFew>(B, upr, p, st);
+}
+}  // namespace
+
+hif4_status launch_gemv(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,
+                        void* workspace, cudaStream_t st) {
+  GemvParams p{};
+  p.A = static_cast<const uint32_t*>(A);
+  if (!gemv_params(p, C, M, N, K, ldc, workspace)) return HIF4_ERR_SHAPE;
+  if (!p.error_word) return HIF4_ERR_CUDA;
+  const int m_pad = M <= 8 ? 8 : 16;
+  const int64_t upr = K / kUnitElems;
+  const int64_t prep = static_cast<int64_t>(m_pad) * upr;
+  gemv_prepare_tokens_kernel<<<static_cast<unsigned>(ceil_div64(prep, 128)), 128, 0, st>>>(p.A, p.M, m_pad, upr, p.tokens);
+  note_launch();
+  if (cudaGetLastError() != cudaSuccess) return HIF4_ERR_CUDA;
+  return launch_gemv_stream(B, p, m_pad, upr, st);
+}
+
+bool gemv_linear_supported(const void* X, int64_t ld_x, const void* B, int64_t M, int64_t N, int64_t K) {
+  return M >= 1 && M <= kGemvMaxM && gemm_tc_supported(B, B, N, N, N, K) && (reinterpret_cast<uintptr_t>(X) & 15u) == 0 &&
+         ld_x >= K && (ld_x * 2) % 16 == 0;
+}
+
+hif4_status launch_gemv_linear_bf16(const void* X, int64_t ld_x, int rha, const void* B, float* C, int64_t M, int64_t N,
+                                    int64_t K, int64_t ldc, void* workspace, cudaStream_t st) {
+  GemvParams p{};
+  if (!gemv_params(p, C, M, N, K, ldc, workspace)) return HIF4_ERR_SHAPE;
+  if (!p.error_word) return HIF4_ERR_CUDA;
+  const int m_pad = M <= 8 ? 8 : 16;
+  const int64_t upr = K / kUnitElems;
+  const int64_t threads = 2 * static_cast<int64_t>(m_pad) * upr;
+  const unsigned blocks = static_cast<unsigned>(ceil_div64(threads, 128));
+  const uint16_t* x = static_cast<const uint16_t*>(X);
+  if (rha) gemv_quantize_tokens_kernel<true><<<blocks, 128, 0, st>>>(x, ld_x, p.M, m_pad, upr, p.tokens);
+  else gemv_quantize_tokens_kernel<false><<<blocks, 128, 0, st>>>(x, ld_x, p.M, m_pad, upr, p.tokens);
+  note_launch();
+  if (cudaGetLastError() != cudaSuccess) return HIF4_ERR_CUDA;
+  return launch_gemv_stream(B, p, m_pad, upr, st);
 }
 
 }  // namespace hif4

@@ -440,3 +440,25 @@ def test_linear_is_quantize_then_gemm(hif4, M, N, K, dtype):
     ref, refabs = oracle.gemm_f64(oracle.quantize(src), w.cpu().numpy(), nthreads=8)
     assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - ref) <= TOL * refabs + 1e-300)
     assert hif4.lib.hif4_linear(x.data_ptr(), 0, K, w.data_ptr(), y.data_ptr(), M, N, K, N, 0, None, 0, None) == 5
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("M,N,K", [(1, 4096, 4096), (16, 1000, 1024), (7, 260, 256), (9, 64, 2304), (16, 14336, 4096)])
+def test_linear_with_few_rows_quantizes_inside_the_token_preparation(hif4, M, N, K, mode):
+    """M <= 16 rows of BF16 activations: hif4_linear runs two kernels (quantize-and-decode of the tokens, weight
+    streaming) instead of three and gives exactly the bits of hif4_quantize followed by hif4_gemm -- on a strided
+    source with spikes, a NaN and an Inf, in both rounding modes."""
+    g = torch.Generator(device="cuda"); g.manual_seed(M * 3 + N + K + mode)
+    wide = torch.randn(M, K + 64, generator=g, device="cuda").to(torch.bfloat16)
+    x = wide[:, 64:]                                      # row stride K + 64
+    x[0, 5] = 1000.0
+    if M > 2:
+        x[1, 70] = float("nan")
+        x[2, 129] = float("-inf")
+    w = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
+    before = hif4.launch_count()
+    y = hif4.hif4_linear(x, w, mode=mode)
+    assert hif4.launch_count() - before == 2
+    want = hif4.hif4_gemm(hif4.hif4_quantize(x, mode), w)
+    assert torch.equal(y.view(torch.int32), want.view(torch.int32)), "fused token preparation differs from quantize + GEMM"
+    assert hif4.hif4_last_device_status() == 0
