@@ -144,7 +144,8 @@ def run_cuda(args):
         xq[(M, K, N)] = torch.empty(M, K // 64, 36, dtype=torch.uint8, device=dev)
         cs[(M, K, N)] = torch.empty(M, N, dtype=torch.float32, device=dev)
     # one scratch buffer for the GEMM workspaces (stream-ordered reuse)
-    ws = torch.empty(max(max(hif4.hif4_gemm_workspace(M, N, K) for (M, K, N, _) in SHAPES), 256), dtype=torch.uint8, device=dev)
+    ws = torch.empty(max(max(max(hif4.hif4_gemm_workspace(M, N, K), hif4.hif4_linear_workspace(M, N, K) if M <= 16 else 0)
+                             for (M, K, N, _) in SHAPES), 256), dtype=torch.uint8, device=dev)
     torch.cuda.synchronize()
 
     stream = torch.cuda.current_stream()
@@ -168,6 +169,12 @@ def run_cuda(args):
                 e2.record(stream)
                 events.append(((M, K, N), e0, e1, e2))
 
+    def run_linears(shapes):
+        """The same work through the one-call linear layer (quantize + GEMM): for M <= 16 the activations are
+        quantized inside the token preparation of the weight-streaming kernel, one launch fewer per linear."""
+        for (M, K, N, name) in shapes:
+            hif4.hif4_linear(acts[(M, K)], weights[(K, N)], out=cs[(M, K, N)], workspace=ws)
+
     def barrier():
         dp.barrier()
         torch.cuda.synchronize()
@@ -176,6 +183,7 @@ def run_cuda(args):
     sampler.start()
     for _ in range(max(args.warmup, 3)):
         run_shapes(SHAPES)
+    run_linears(small)
     barrier()
 
     # The launches of the decode-shaped linears are captured once into two CUDA graphs (M=1, M=16) and
@@ -187,7 +195,7 @@ def run_cuda(args):
             n0 = hif4.launch_count()
             graphs[gi] = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graphs[gi]):
-                run_shapes(groups[gi])
+                run_linears(groups[gi])
             graph_launches += hif4.launch_count() - n0
         torch.cuda.synchronize()
 
@@ -196,7 +204,7 @@ def run_cuda(args):
             if gi in graphs:
                 graphs[gi].replay()
             elif gi in (0, 2):
-                run_shapes(shapes)
+                run_linears(shapes)
             else:
                 run_shapes(shapes, events)
 
@@ -270,8 +278,9 @@ def run_cuda(args):
                    "l2": "no flush: the step order (M=1 linears, two prefill linears, M=16 linears, two prefill linears) "
                          "touches > 126 MB (L2) between two uses of any tensor; per_shape rows with M <= 16 come from "
                          "a separate pass that writes 256 MB before each linear",
-                   "launch": ("decode-shaped linears replayed from two CUDA graphs per step, prefill linears launched directly"
-                              if graphs else "every kernel launched directly"),
+                   "launch": ("decode-shaped linears (hif4_linear, two kernels each) replayed from two CUDA graphs per step, "
+                              "prefill linears (hif4_quantize + hif4_gemm) launched directly"
+                              if graphs else "every kernel launched directly (hif4_linear for M <= 16, hif4_quantize + hif4_gemm for M = 4096)"),
                    "parallelism": f"dp{world} (independent token batches, no collective)"},
         "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "per_shape": table,
     }

@@ -73,29 +73,29 @@ def test_llama_linears_all_m(hif4):
 
 
 def test_llama_decode_linears_replayed_from_a_cuda_graph(hif4):
-    """The benchmark replays the M = 1 and M = 16 linears (quantize + GEMM, shared workspace) from CUDA graphs:
-    same launches, captured once; the replayed results are checked like the direct ones and are identical to them."""
+    """The benchmark replays the M = 1 and M = 16 linears (hif4_linear: token quantization + preparation, then
+    weight streaming; shared workspace) from CUDA graphs: the same launches, captured once.  The replayed results
+    are identical to hif4_quantize + hif4_gemm launched directly and are checked against the oracle like them."""
     shapes = [(M, K, N) for M in (1, 16) for (_, K, N) in wl.LLAMA3_8B_LINEARS]
     weights = {(K, N): hif4.hif4_quantize(wl.gaussian(N, K, 0.02, seed=2000 + N + K, device="cuda"))
                for (_, K, N) in wl.LLAMA3_8B_LINEARS}
     acts = {(M, K): wl.llama_activations(M, K, seed=1002 + M + K, device="cuda") for (M, K, _) in shapes}
-    xq = {sh: torch.empty(sh[0], sh[1] // 64, 36, dtype=torch.uint8, device="cuda") for sh in shapes}
+    xq = {sh: hif4.hif4_quantize(acts[(sh[0], sh[1])]) for sh in shapes}
     cs = {sh: torch.empty(sh[0], sh[2], dtype=torch.float32, device="cuda") for sh in shapes}
-    ws = torch.empty(max(max(hif4.hif4_gemm_workspace(M, N, K) for (M, K, N) in shapes), 256), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(max(max(hif4.hif4_linear_workspace(M, N, K) for (M, K, N) in shapes), 256), dtype=torch.uint8, device="cuda")
+    direct = {sh: hif4.hif4_gemm(xq[sh], weights[(sh[1], sh[2])]) for sh in shapes}
 
     def run():
         for (M, K, N) in shapes:
-            hif4.hif4_quantize(acts[(M, K)], out=xq[(M, K, N)])
-            hif4.hif4_gemm(xq[(M, K, N)], weights[(K, N)], out=cs[(M, K, N)], workspace=ws)
+            hif4.hif4_linear(acts[(M, K)], weights[(K, N)], out=cs[(M, K, N)], workspace=ws)
 
     run()                                               # direct launches (also the one-time kernel attributes)
     torch.cuda.synchronize()
-    direct = {sh: c.clone() for sh, c in cs.items()}
     graph = torch.cuda.CUDAGraph()
     before = hif4.launch_count()
     with torch.cuda.graph(graph):
         run()
-    assert hif4.launch_count() - before == 3 * len(shapes), "quantize + token preparation + streaming kernel per linear"
+    assert hif4.launch_count() - before == 2 * len(shapes), "token preparation + streaming kernel per linear"
     for c in cs.values():
         c.fill_(-7.0)
     for _ in range(3):
@@ -104,7 +104,7 @@ def test_llama_decode_linears_replayed_from_a_cuda_graph(hif4):
     assert hif4.hif4_last_device_status() == 0
     for sh in shapes:
         M, K, N = sh
-        assert torch.equal(cs[sh], direct[sh]), f"replayed {sh} differs from the direct launch"
+        assert torch.equal(cs[sh], direct[sh]), f"replayed {sh} differs from hif4_quantize + hif4_gemm"
         _sampled_entries(hif4, xq[sh], weights[(K, N)], cs[sh], f"graph replay {sh}", n=100, seed=M + N)
 
 
