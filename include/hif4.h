@@ -87,6 +87,20 @@ size_t hif4_packed_bytes(int64_t rows, int64_t cols);
 hif4_status hif4_quantize(const void* src, hif4_dtype dt, int64_t rows, int64_t cols,
                           int64_t ld_src, void* dst_units, hif4_round mode, void* stream);
 
+/* hif4_quantize_transposed -- the same conversion with the units running down the columns: unit r of
+ * column c holds src[64 r .. 64 r + 63][c], i.e. dst is hif4_quantize of the transposed matrix without the
+ * transpose ever being written.  (Algorithm 1 converts "a vector of 64" values and does not say how the
+ * vector lies in memory; Eq. 3 needs both GEMM operands cut along the contraction dimension, so a matrix
+ * that is contracted along its rows -- a weight kept as [K, N], or any operand of a transposed product --
+ * is quantized this way.)
+ *   src        device, [rows, cols] BF16, row stride `ld_src` elements (>= cols), rows 16-byte aligned;
+ *              rows must be a multiple of 64, cols a multiple of 8.
+ *   dst_units  device, cols*(rows/64) units, column-major in the sense above ([cols, rows/64, 36 bytes]),
+ *              4-byte aligned.  Fully overwritten.
+ * Only HIF4_BF16 sources are built (others return HIF4_ERR_UNSUPPORTED).  */
+hif4_status hif4_quantize_transposed(const void* src, hif4_dtype dt, int64_t rows, int64_t cols,
+                                     int64_t ld_src, void* dst_units, hif4_round mode, void* stream);
+
 /* hif4_dequantize -- Eq. 2 for every element; exact in BF16 and FP32.
  *   src_units  device, rows*(cols/64) units, 4-byte aligned.
  *   dst        device, [rows, cols] of `dt`, row stride `ld_dst` elements (>= cols), rows 16-byte

@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = [
     "hif4_packed_bytes", "hif4_quantize", "hif4_dequantize", "hif4_gemm_workspace", "hif4_gemm",
     "hif4_grouped_gemm_workspace", "hif4_grouped_gemm", "hif4_last_device_status", "hif4_status_string",
     "hif4_launch_count", "hif4_set_gemm_path", "hif4_grouped_gemm_noalloc", "hif4_grouped_gemm_noalloc_capacity",
-    "hif4_linear", "hif4_linear_workspace",
+    "hif4_linear", "hif4_linear_workspace", "hif4_quantize_transposed",
 ]
 
 
@@ -45,6 +45,8 @@ def _load() -> ctypes.CDLL:
     L.hif4_packed_bytes.argtypes = [i64, i64]
     L.hif4_quantize.restype = ci
     L.hif4_quantize.argtypes = [vp, ci, i64, i64, i64, vp, ci, vp]
+    L.hif4_quantize_transposed.restype = ci
+    L.hif4_quantize_transposed.argtypes = [vp, ci, i64, i64, i64, vp, ci, vp]
     L.hif4_dequantize.restype = ci
     L.hif4_dequantize.argtypes = [vp, i64, i64, vp, ci, i64, vp]
     L.hif4_gemm_workspace.restype = ci
@@ -128,6 +130,21 @@ def hif4_quantize(src: torch.Tensor, mode: int = HIF4_RNE, out: Optional[torch.T
     ld = src.stride(0) if rows > 1 else max(cols, src.stride(0))
     _check("hif4_quantize", lib.hif4_quantize(src.data_ptr(), _dtype_code(src.dtype), rows, cols, ld,
                                               out.data_ptr(), mode, _stream(stream)))
+    return out
+
+
+def hif4_quantize_transposed(src: torch.Tensor, mode: int = HIF4_RNE, out: Optional[torch.Tensor] = None,
+                             stream=None) -> torch.Tensor:
+    """[rows, cols] BF16 -> uint8 units [cols, rows // 64, 36]: the units of src.T without transposing."""
+    _need_cuda(src, out)
+    assert src.dim() == 2 and src.stride(1) == 1
+    rows, cols = src.shape
+    if out is None:
+        out = torch.empty((cols, rows // UNIT_ELEMS if rows % UNIT_ELEMS == 0 else 0, UNIT_BYTES),
+                          dtype=torch.uint8, device=src.device)
+    ld = src.stride(0) if rows > 1 else max(cols, src.stride(0))
+    _check("hif4_quantize_transposed", lib.hif4_quantize_transposed(src.data_ptr(), _dtype_code(src.dtype), rows, cols, ld,
+                                                                    out.data_ptr(), mode, _stream(stream)))
     return out
 
 

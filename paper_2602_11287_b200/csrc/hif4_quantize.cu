@@ -94,6 +94,61 @@ quantize_bf16_kernel(const uint16_t* __restrict__ src, int64_t n_units, int64_t 
   }
 }
 
+// ----------------------------------------------------------------------------- BF16 quantizer, units down the columns
+// One block converts a tile of 64 rows x 128 columns: the rows are read as they lie (256 bytes each), staged in
+// shared memory, and each pair of lanes then takes two neighbouring columns (one 32-bit word per row) as its
+// two units, lane l again the level-2 groups l, l + 2, l + 4, l + 6 of both.  Same encoder as above, so the units
+// are those of hif4_quantize on the transposed matrix.
+constexpr int kTileCols = 128;
+constexpr int kTilePitchWords = kTileCols / 2 + 1;        // 32-bit words per staged row: column reads of consecutive rows hit different banks
+
+template <bool kRHA>
+__global__ void __launch_bounds__(128)
+quantize_bf16_transposed_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t cols, int64_t ld_src,
+                                uint32_t* __restrict__ dst) {
+  __shared__ uint32_t tile[kUnitElems * kTilePitchWords];
+  // consecutive blocks take consecutive row tiles of the same columns: their units are neighbours in dst
+  const int64_t c0 = static_cast<int64_t>(blockIdx.y) * kTileCols;
+  const int64_t r0 = static_cast<int64_t>(blockIdx.x) * kUnitElems;
+  // 64 rows x 16 chunks of 8 elements; a chunk is inside the matrix or outside as a whole (cols % 8 == 0)
+  for (int i = threadIdx.x; i < kUnitElems * (kTileCols / 8); i += blockDim.x) {
+    const int r = i >> 4, ch = i & 15;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (c0 + 8 * ch < cols) v = ld_stream(reinterpret_cast<const uint4*>(src + (r0 + r) * ld_src + c0 + 8 * ch));
+    uint32_t* t = tile + r * kTilePitchWords + 4 * ch;
+    t[0] = v.x; t[1] = v.y; t[2] = v.z; t[3] = v.w;
+  }
+  __syncthreads();
+  const int l = threadIdx.x & 1, cp = threadIdx.x >> 1;     // columns 2 cp and 2 cp + 1 of the tile
+  uint4 even[4], odd[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const uint32_t* p = tile + (8 * (l + 2 * c)) * kTilePitchWords + cp;           // rows 8 g .. 8 g + 7, both columns
+    uint32_t e[4], o[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t a = p[(2 * k) * kTilePitchWords], b2 = p[(2 * k + 1) * kTilePitchWords];
+      e[k] = prmt(a, b2, 0x5410u);                          // low halves: the even column of rows 2k, 2k + 1
+      o[k] = prmt(a, b2, 0x7632u);                          // high halves: the odd column
+    }
+    even[c] = make_uint4(e[0], e[1], e[2], e[3]);
+    odd[c] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+  const int64_t units_per_col = rows / kUnitElems;
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    uint32_t codes[4], meta;
+    encode_unit_bf16_pair<kRHA>(half ? odd : even, l, codes, meta);
+    const int64_t col = c0 + 2 * cp + half;
+    if (col < cols) {
+      uint32_t* out = dst + (col * units_per_col + blockIdx.x) * kUnitWords;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) st_stream(out + 1 + 2 * c + l, codes[c]);
+      if (l == 0) st_stream(out, meta);
+    }
+  }
+}
+
 // ----------------------------------------------------------------------------- FP32 quantizer
 // Same steps as above in FP32 arithmetic: (1/7) and the reciprocal table are the nearest FP32 values,
 // every product is a single mul.rn.f32.  One level-3 group (4 elements): micro-exponent from the peak
@@ -328,6 +383,27 @@ extern "C" hif4_status hif4_quantize(const void* src, hif4_dtype dt, int64_t row
   } else {
     launch_quantize_fp32(static_cast<const __half*>(src), rha, contig, grid, st, n_units, upr, ld_src, dst);
   }
+  note_launch();
+  return launch_status();
+}
+
+extern "C" hif4_status hif4_quantize_transposed(const void* src, hif4_dtype dt, int64_t rows, int64_t cols,
+                                                int64_t ld_src, void* dst_units, hif4_round mode, void* stream) {
+  if (dt != HIF4_BF16 && dt != HIF4_FP32 && dt != HIF4_FP16) return HIF4_ERR_DTYPE;
+  if (mode != HIF4_RNE && mode != HIF4_RHA) return HIF4_ERR_DTYPE;
+  if (rows < 0 || cols < 0 || rows % kUnitElems != 0 || cols % 8 != 0 || ld_src < cols) return HIF4_ERR_SHAPE;
+  if (rows == 0 || cols == 0) return HIF4_OK;
+  if (!src || !dst_units) return HIF4_ERR_NULL;
+  if (dt != HIF4_BF16) return HIF4_ERR_UNSUPPORTED;
+  if (!aligned(src, 16) || (static_cast<size_t>(ld_src) * 2) % 16 != 0 || !aligned(dst_units, 4)) return HIF4_ERR_ALIGN;
+  const int64_t col_tiles = ceil_div64(cols, kTileCols), row_tiles = rows / kUnitElems;
+  if (row_tiles > 0x7FFFFFFFll || col_tiles > 65535) return HIF4_ERR_SHAPE;
+  const dim3 grid(static_cast<unsigned>(row_tiles), static_cast<unsigned>(col_tiles));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const uint16_t* x = static_cast<const uint16_t*>(src);
+  uint32_t* dst = static_cast<uint32_t*>(dst_units);
+  if (mode == HIF4_RHA) quantize_bf16_transposed_kernel<true><<<grid, 128, 0, st>>>(x, rows, cols, ld_src, dst);
+  else quantize_bf16_transposed_kernel<false><<<grid, 128, 0, st>>>(x, rows, cols, ld_src, dst);
   note_launch();
   return launch_status();
 }

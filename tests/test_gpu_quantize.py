@@ -205,3 +205,42 @@ def test_quantize_fp16_source(hif4, mode):
     w = hif4.hif4_quantize((torch.randn(96, 512, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
     y = hif4.hif4_linear(x16, w, mode=mode)
     assert torch.equal(y, hif4.hif4_gemm(hif4.hif4_quantize(x16, mode), w))
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_quantize_transposed_is_quantize_of_the_transpose(hif4, mode):
+    """Units down the columns: bit-identical to the oracle's Algorithm 1 on the transposed matrix, for ragged column
+    counts, a strided source, random bit patterns (NaN and Inf included) and the workload mix."""
+    rng = np.random.default_rng(500 + mode)
+    cases = []
+    for (rows, cols) in ((64, 8), (128, 72), (640, 1000), (1024, 2048)):
+        expo = rng.integers(100, 150, size=(1, cols), dtype=np.uint32)                 # per column: base exponent
+        mant = rng.integers(0, 1 << 7, size=(rows, cols), dtype=np.uint32)
+        sign = rng.integers(0, 2, size=(rows, cols), dtype=np.uint32) << 15
+        spread = rng.integers(0, 7, size=(rows, cols), dtype=np.uint32)
+        cases.append((sign | ((expo - spread) << 7) | mant).astype(np.uint16))
+    cases.append(rng.integers(0, 1 << 16, size=(256, 512), dtype=np.uint32).astype(np.uint16))      # every kind of value
+    cases.append(wl.bf16_to_u16_numpy(wl.quantize_sweep(2 ** 20, device="cuda")))                   # [256, 4096] workload mix
+    for bits in cases:
+        rows, cols = bits.shape
+        x = wl.u16_numpy_to_bf16(bits, "cuda")
+        out = torch.full((cols + 2, rows // 64, 36), 0xCD, dtype=torch.uint8, device="cuda")
+        hif4.hif4_quantize_transposed(x, mode, out=out[1:cols + 1])
+        want = oracle.quantize(np.ascontiguousarray(bits.T), mode, nthreads=8)
+        _compare_units(out[1:cols + 1].cpu().numpy(), want, f"transposed {rows}x{cols} mode {mode}")
+        assert (out[0] == 0xCD).all() and (out[cols + 1] == 0xCD).all()
+        assert torch.equal(out[1:cols + 1], hif4.hif4_quantize(x.t().contiguous(), mode)), "differs from quantizing the transpose"
+    # strided source
+    wide = wl.u16_numpy_to_bf16(cases[2], "cuda")
+    view = wide[:, 8:808]
+    got = hif4.hif4_quantize_transposed(view, mode).cpu().numpy()
+    _compare_units(got, oracle.quantize(np.ascontiguousarray(cases[2][:, 8:808].T), mode, nthreads=8), "transposed, strided")
+    # argument checks
+    with pytest.raises(hif4.Hif4Error) as ei:
+        hif4.hif4_quantize_transposed(torch.zeros(100, 64, dtype=torch.bfloat16, device="cuda"))
+    assert ei.value.code == 2                                                                      # rows % 64
+    with pytest.raises(hif4.Hif4Error) as ei:
+        hif4.hif4_quantize_transposed(torch.zeros(64, 64, dtype=torch.float32, device="cuda"))
+    assert ei.value.code == 8                                                                      # BF16 only
+    assert hif4.hif4_quantize_transposed(torch.zeros(0, 64, dtype=torch.bfloat16, device="cuda")).shape == (64, 0, 36)
+    assert hif4.hif4_last_device_status() == 0
