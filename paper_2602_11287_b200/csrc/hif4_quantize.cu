@@ -26,7 +26,8 @@ namespace hif4 {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kUnroll = 4;
+// units per 8-lane group and pass of the dequantizer: more loads in flight pay for BF16 output, not for FP32
+constexpr int kUnrollDeqBf16 = 8, kUnrollDeqFp32 = 8;
 
 // ----------------------------------------------------------------------------- streaming loads and stores
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
@@ -278,21 +279,26 @@ quantize_fp32_kernel(const Src* __restrict__ src, int64_t n_units, int64_t upr, 
 }
 
 // ----------------------------------------------------------------------------- dequantizer (Eq. 2)
-// 8 lanes per unit; lane j decodes code word j (elements 8j..8j+7).  Each value is
-// m * (4+M) * 2^(E-48-4+e8+e16): an integer below 64 times a power of two, exact in FP32 and BF16.
+// BF16 output: 8 lanes per unit, lane j decodes code word j (elements 8j..8j+7, 16 bytes of output).  FP32 output:
+// 16 lanes per unit, lane k decodes half k & 1 of code word k >> 1 (4 elements, again 16 bytes of output), so that
+// every store instruction of a warp writes whole, consecutive sectors.  Each value is
+// m * (4+M) * 2^(E-48-4+e8+e16): an integer below 64 times a power of two, exact in BF16 (and so in FP32).
 template <bool kBF16Out, bool kContig>
 __global__ void __launch_bounds__(kThreads)
 dequantize_kernel(const uint32_t* __restrict__ src, int64_t n_units, int64_t upr, int64_t ld_dst,
                   void* __restrict__ dst) {
+  constexpr int kLanes = kBF16Out ? 8 : 16;                   // lanes per unit
+  constexpr int kUnroll = kBF16Out ? kUnrollDeqBf16 : kUnrollDeqFp32;
   const int lane = threadIdx.x & 31;
-  const int j = lane & 7;
+  const int k = lane & (kLanes - 1);
+  const int j = kBF16Out ? k : k >> 1;                        // code word
   const int64_t warp = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) >> 5;
-  const int64_t first = warp * (4 * kUnroll) + (lane >> 3);
+  const int64_t first = warp * ((32 / kLanes) * kUnroll) + lane / kLanes;
 
   uint32_t meta[kUnroll], word[kUnroll];
 #pragma unroll
   for (int i = 0; i < kUnroll; ++i) {
-    const int64_t u = first + 4 * i;
+    const int64_t u = first + (32 / kLanes) * i;
     meta[i] = 0; word[i] = 0;
     if (u < n_units) {
       meta[i] = __ldg(src + u * kUnitWords);
@@ -301,37 +307,38 @@ dequantize_kernel(const uint32_t* __restrict__ src, int64_t n_units, int64_t upr
   }
 #pragma unroll
   for (int i = 0; i < kUnroll; ++i) {
-    const int64_t u = first + 4 * i;
+    const int64_t u = first + (32 / kLanes) * i;
     if (u >= n_units) continue;
     const uint32_t byte = meta[i] & 0xFFu;
     const uint32_t e8 = (meta[i] >> (8 + j)) & 1u;
     const uint32_t e16a = (meta[i] >> (16 + 2 * j)) & 1u, e16b = (meta[i] >> (17 + 2 * j)) & 1u;
-    // (4 + M) * 2^(E - 48 - 4 + shift) as FP32 bits: exponent field (byte >> 2) - 52 + 127 + 2 + shift, the
-    // three bits of 4 + M on top of the mantissa (1.00, 1.01, 1.10, 1.11)
-    const uint32_t sbits = (((byte >> 2) + 77u + e8) << 23) | ((byte & 3u) << 21);
-    const float sa = __uint_as_float(sbits + (e16a << 23)), sb = __uint_as_float(sbits + (e16b << 23));
-    // m * s without an integer-to-float conversion: (2^23 + m) * s - 2^23 * s in one fused multiply-add
-    // (the exact product is rounded once, and m * s is representable)
-    const float na = -8388608.0f * sa, nb = -8388608.0f * sb;
-    uint32_t bits[8];
+    // Packed BF16 arithmetic, two elements per instruction: S = E6M2 / 4 * 2^shift as BF16 bits is
+    // ((byte + 308) << 5) + (shift << 7); (128 + m) * S - 128 * S in one fused multiply-add is m * S exactly; the
+    // sign bit goes on afterwards so that a negative zero stays negative.
+    const uint32_t base = (byte + 308u) << 5;
+    const uint32_t S = (base + ((e8 + e16a) << 7)) | ((base + ((e8 + e16b) << 7)) << 16);   // (elements 0..3, elements 4..7)
+    const uint32_t O = S + 0x83808380u;                                                     // -128 S
+    const uint32_t w = word[i];
+    uint32_t r[4];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const uint32_t c = word[i] >> (4 * e);
-      const float val = __fmaf_rn(__uint_as_float((c & 7u) | 0x4B000000u), e < 4 ? sa : sb, e < 4 ? na : nb);
-      bits[e] = byte == 0xFFu ? 0x7FC00000u : (__float_as_uint(val) | ((c & 8u) << 28));
+    for (int e = 0; e < 4; ++e) {                                                           // elements e and e + 4
+      const uint32_t c = w >> (4 * e);
+      r[e] = fma_bf16x2((c & 0x00070007u) | 0x43004300u, S, O) | ((c << 12) & 0x80008000u);
+      if (byte == 0xFFu) r[e] = 0x7FC07FC0u;                                                // NaN unit
     }
-    const int64_t off = unit_offset<kContig>(u, upr, ld_dst) + 8 * j;
     if (kBF16Out) {
+      const int64_t off = unit_offset<kContig>(u, upr, ld_dst) + 8 * j;
       uint4 o;
-      o.x = (bits[0] >> 16) | (bits[1] & 0xFFFF0000u);
-      o.y = (bits[2] >> 16) | (bits[3] & 0xFFFF0000u);
-      o.z = (bits[4] >> 16) | (bits[5] & 0xFFFF0000u);
-      o.w = (bits[6] >> 16) | (bits[7] & 0xFFFF0000u);
+      o.x = prmt(r[0], r[1], 0x5410u);          // elements 0, 1
+      o.y = prmt(r[2], r[3], 0x5410u);          // elements 2, 3
+      o.z = prmt(r[0], r[1], 0x7632u);          // elements 4, 5
+      o.w = prmt(r[2], r[3], 0x7632u);          // elements 6, 7
       st_stream(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + off), o);
-    } else {
-      uint4* p = reinterpret_cast<uint4*>(static_cast<float*>(dst) + off);
-      st_stream(p, make_uint4(bits[0], bits[1], bits[2], bits[3]));
-      st_stream(p + 1, make_uint4(bits[4], bits[5], bits[6], bits[7]));
+    } else {                                    // a BF16 widens to FP32 by appending sixteen zero bits
+      const int64_t off = unit_offset<kContig>(u, upr, ld_dst) + 4 * k;
+      const uint4 o = (k & 1) ? make_uint4(r[0] & 0xFFFF0000u, r[1] & 0xFFFF0000u, r[2] & 0xFFFF0000u, r[3] & 0xFFFF0000u)
+                              : make_uint4(r[0] << 16, r[1] << 16, r[2] << 16, r[3] << 16);
+      st_stream(reinterpret_cast<uint4*>(static_cast<float*>(dst) + off), o);
     }
   }
 }
@@ -420,7 +427,7 @@ extern "C" hif4_status hif4_dequantize(const void* src_units, int64_t rows, int6
   const int64_t upr = cols / kUnitElems;
   const int64_t n_units = rows * upr;
   const bool contig = ld_dst == cols;
-  const int64_t blocks = ceil_div64(n_units, (kThreads / 32) * kUnroll * 4);
+  const int64_t blocks = ceil_div64(n_units, (kThreads / 32) * (dt == HIF4_BF16 ? kUnrollDeqBf16 * 4 : kUnrollDeqFp32 * 2));
   if (blocks > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const uint32_t* in = static_cast<const uint32_t*>(src_units);
