@@ -139,12 +139,13 @@ extern "C" hif4_status hif4_linear(const void* X, hif4_dtype dt, int64_t ld_x, c
   if (need > 0 && !aligned(workspace, 256)) return HIF4_ERR_ALIGN;
   const size_t x_bytes = round256(hif4_packed_bytes(M, K));
   uint8_t* x_units = static_cast<uint8_t*>(workspace);
-  // Few rows of BF16 activations: quantized and decoded inside the token preparation of the weight-streaming
-  // kernel (same encoder code, so the same bits), one launch fewer and no packed round trip.
-  if (dt == HIF4_BF16 && (mode == HIF4_RNE || mode == HIF4_RHA) && K > 0 && (g_gemm_path == 0 || g_gemm_path == 4) && X &&
-      W_units && Y && ldy >= N && aligned(W_units, 4) && aligned(Y, 4) && gemv_linear_supported(X, ld_x, W_units, M, N, K))
-    return launch_gemv_linear_bf16(X, ld_x, mode == HIF4_RHA, W_units, Y, M, N, K, ldy, x_units + x_bytes,
-                                   static_cast<cudaStream_t>(stream));
+  // Few rows of activations: quantized and decoded inside the token preparation of the weight-streaming kernel
+  // (same encoder code, so the same bits), one launch fewer and no packed round trip.
+  if ((dt == HIF4_BF16 || dt == HIF4_FP32 || dt == HIF4_FP16) && (mode == HIF4_RNE || mode == HIF4_RHA) && K > 0 &&
+      (g_gemm_path == 0 || g_gemm_path == 4) && X && W_units && Y && ldy >= N && aligned(W_units, 4) && aligned(Y, 4) &&
+      gemv_linear_supported(X, dt, ld_x, W_units, M, N, K))
+    return launch_gemv_linear(X, dt, ld_x, mode == HIF4_RHA, W_units, Y, M, N, K, ldy, x_units + x_bytes,
+                              static_cast<cudaStream_t>(stream));
   if (K > 0) {
     const hif4_status q = hif4_quantize(X, dt, M, K, ld_x, x_units, mode, stream);
     if (q != HIF4_OK) return q;

@@ -28,11 +28,11 @@ bool gemv_supported(const void* A, const void* B, int64_t M, int64_t N, int64_t 
 size_t gemv_workspace_bytes(int64_t M, int64_t K);
 hif4_status launch_gemv(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,
                         void* workspace, cudaStream_t st);
-// The same with the activations still in BF16 ([M, K], row stride ld_x elements, 16-byte aligned rows): the
-// token preparation quantizes (Algorithm 1) and decodes in one kernel, the packed units are never written.
-bool gemv_linear_supported(const void* X, int64_t ld_x, const void* B, int64_t M, int64_t N, int64_t K);
-hif4_status launch_gemv_linear_bf16(const void* X, int64_t ld_x, int rha, const void* B, float* C, int64_t M, int64_t N,
-                                    int64_t K, int64_t ldc, void* workspace, cudaStream_t st);
+// The same with the activations not yet quantized ([M, K] of `dt`, row stride ld_x elements, 16-byte aligned rows):
+// the token preparation quantizes (Algorithm 1) and decodes in one kernel, the packed units are never written.
+bool gemv_linear_supported(const void* X, hif4_dtype dt, int64_t ld_x, const void* B, int64_t M, int64_t N, int64_t K);
+hif4_status launch_gemv_linear(const void* X, hif4_dtype dt, int64_t ld_x, int rha, const void* B, float* C, int64_t M,
+                               int64_t N, int64_t K, int64_t ldc, void* workspace, cudaStream_t st);
 size_t grouped_tc_workspace_bytes(int num_groups, int64_t total_rows);
 hif4_status launch_grouped_gemm_tc(const void* A, const void* B, float* C, const int64_t* offsets, int num_groups,
                                    int64_t total_rows, int64_t N, int64_t K, int64_t ldc, void* workspace,

@@ -124,7 +124,7 @@ gemv_prepare_tokens_kernel(const uint32_t* __restrict__ A, int M, int m_pad, int
 
 // The same preparation straight from BF16 activations: Algorithm 1 (the streaming quantizer's own code, two
 // lanes per unit) followed by Eq. 2 of the unit just encoded, without the packed units ever going to memory.
-// Used by the one-call linear layer for M <= 16; the tokens written are bit-identical to quantizing first.
+// Used by the one-call linear layer for M <= 16 BF16 rows; the tokens written are bit-identical to quantizing first.
 template <bool kRHA>
 __global__ void __launch_bounds__(128)
 gemv_quantize_tokens_kernel(const uint16_t* __restrict__ X, int64_t ld_x, int M, int m_pad, int64_t upr,
@@ -154,6 +154,46 @@ gemv_quantize_tokens_kernel(const uint16_t* __restrict__ X, int64_t ld_x, int M,
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
     const int W = l + 2 * c;                             // this lane's code words
+    uint32_t r[4] = {0u, 0u, 0u, 0u};
+    if (n < M) {
+      if (byte == 0xFFu) r[0] = r[1] = r[2] = r[3] = 0x7FC07FC0u;
+      else decode_word_regs(meta, base2, W, codes[c], r);
+    }
+    *reinterpret_cast<uint4*>(dst + W * kTokChunkBytes) = make_uint4(r[0], r[1], r[2], r[3]);
+  }
+}
+
+// The same for FP32 and FP16 activations (Algorithm 1 in FP32 arithmetic, four lanes per unit; the even lanes hold
+// the code words afterwards and decode them).
+template <bool kRHA, typename Src>
+__global__ void __launch_bounds__(128)
+gemv_quantize_tokens32_kernel(const Src* __restrict__ X, int64_t ld_x, int M, int m_pad, int64_t upr,
+                              uint8_t* __restrict__ tokens) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;     // ((token n, unit U), lane l)
+  const int l = static_cast<int>(idx & 3);
+  const int64_t quad = idx >> 2;
+  const bool in_range = quad < static_cast<int64_t>(m_pad) * upr;      // same for the four lanes of a unit
+  const int n = in_range ? static_cast<int>(quad / upr) : 0;
+  const int64_t U = in_range ? quad - static_cast<int64_t>(n) * upr : 0;
+  uint4 v[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) v[c] = make_uint4(0u, 0u, 0u, 0u);
+  if (in_range && n < M) {
+    const Src* src = X + static_cast<int64_t>(n) * ld_x + U * kUnitElems + 4 * l;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) v[c] = load_group_fp32(src + 16 * c);
+  }
+  uint32_t codes[4], meta;
+  encode_unit_fp32_quad<kRHA>(v, l, codes, meta);        // every lane of the warp takes part
+  if (!in_range || (l & 1)) return;
+  const int tiles = m_pad >> 3;
+  uint8_t* dst = tokens + (((U >> 2) * tiles + (n >> 3)) * 8) * kTokChunkBytes + ((n & 7) * 4 + (U & 3)) * 16;
+  const uint32_t byte = meta & 0xFFu;
+  const uint32_t base2 = byte * 0x00200020u + 0x26802680u;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const int W = (l >> 1) + 2 * c;                      // this lane's code words
     uint32_t r[4] = {0u, 0u, 0u, 0u};
     if (n < M) {
       if (byte == 0xFFu) r[0] = r[1] = r[2] = r[3] = 0x7FC07FC0u;
@@ -446,23 +486,34 @@ hif4_status launch_gemv(const void* A, const void* B, float* C, int64_t M, int64
   return launch_gemv_stream(B, p, m_pad, upr, st);
 }
 
-bool gemv_linear_supported(const void* X, int64_t ld_x, const void* B, int64_t M, int64_t N, int64_t K) {
+bool gemv_linear_supported(const void* X, hif4_dtype dt, int64_t ld_x, const void* B, int64_t M, int64_t N, int64_t K) {
+  const int64_t esz = dt == HIF4_FP32 ? 4 : 2;
   return M >= 1 && M <= kGemvMaxM && gemm_tc_supported(B, B, N, N, N, K) && (reinterpret_cast<uintptr_t>(X) & 15u) == 0 &&
-         ld_x >= K && (ld_x * 2) % 16 == 0;
+         ld_x >= K && (ld_x * esz) % 16 == 0;
 }
 
-hif4_status launch_gemv_linear_bf16(const void* X, int64_t ld_x, int rha, const void* B, float* C, int64_t M, int64_t N,
-                                    int64_t K, int64_t ldc, void* workspace, cudaStream_t st) {
+hif4_status launch_gemv_linear(const void* X, hif4_dtype dt, int64_t ld_x, int rha, const void* B, float* C, int64_t M,
+                               int64_t N, int64_t K, int64_t ldc, void* workspace, cudaStream_t st) {
   GemvParams p{};
   if (!gemv_params(p, C, M, N, K, ldc, workspace)) return HIF4_ERR_SHAPE;
   if (!p.error_word) return HIF4_ERR_CUDA;
   const int m_pad = M <= 8 ? 8 : 16;
   const int64_t upr = K / kUnitElems;
-  const int64_t threads = 2 * static_cast<int64_t>(m_pad) * upr;
-  const unsigned blocks = static_cast<unsigned>(ceil_div64(threads, 128));
-  const uint16_t* x = static_cast<const uint16_t*>(X);
-  if (rha) gemv_quantize_tokens_kernel<true><<<blocks, 128, 0, st>>>(x, ld_x, p.M, m_pad, upr, p.tokens);
-  else gemv_quantize_tokens_kernel<false><<<blocks, 128, 0, st>>>(x, ld_x, p.M, m_pad, upr, p.tokens);
+  const int lanes = dt == HIF4_BF16 ? 2 : 4;             // lanes per unit of the encoder
+  const unsigned blocks = static_cast<unsigned>(ceil_div64(lanes * static_cast<int64_t>(m_pad) * upr, 128));
+  if (dt == HIF4_BF16) {
+    const uint16_t* x = static_cast<const uint16_t*>(X);
+    if (rha) gemv_quantize_tokens_kernel<true><<<blocks, 128, 0, st>>>(x, ld_x, p.M, m_pad, upr, p.tokens);
+    else gemv_quantize_tokens_kernel<false><<<blocks, 128, 0, st>>>(x, ld_x, p.M, m_pad, upr, p.tokens);
+  } else if (dt == HIF4_FP32) {
+    const float* x = static_cast<const float*>(X);
+    if (rha) gemv_quantize_tokens32_kernel<true, float><<<blocks, 128, 0, st>>>(x, ld_x, p.M, m_pad, upr, p.tokens);
+    else gemv_quantize_tokens32_kernel<false, float><<<blocks, 128, 0, st>>>(x, ld_x, p.M, m_pad, upr, p.tokens);
+  } else {
+    const __half* x = static_cast<const __half*>(X);
+    if (rha) gemv_quantize_tokens32_kernel<true, __half><<<blocks, 128, 0, st>>>(x, ld_x, p.M, m_pad, upr, p.tokens);
+    else gemv_quantize_tokens32_kernel<false, __half><<<blocks, 128, 0, st>>>(x, ld_x, p.M, m_pad, upr, p.tokens);
+  }
   note_launch();
   if (cudaGetLastError() != cudaSuccess) return HIF4_ERR_CUDA;
   return launch_gemv_stream(B, p, m_pad, upr, st);

@@ -30,13 +30,6 @@ constexpr int kThreads = 256;
 constexpr int kUnrollDeqBf16 = 8, kUnrollDeqFp32 = 8;
 
 // ----------------------------------------------------------------------------- streaming loads and stores
-__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
-  uint4 v;
-  asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
-  return v;
-}
 __device__ __forceinline__ void st_stream(uint32_t* p, uint32_t v) {
   asm volatile("st.global.cs.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
@@ -151,47 +144,10 @@ quantize_bf16_transposed_kernel(const uint16_t* __restrict__ src, int64_t rows, 
 }
 
 // ----------------------------------------------------------------------------- FP32 quantizer
-// Same steps as above in FP32 arithmetic: (1/7) and the reciprocal table are the nearest FP32 values,
-// every product is a single mul.rn.f32.  One level-3 group (4 elements): micro-exponent from the peak
-// of the products (e8 is passed in), codes as four nibbles in the low 16 bits.
-template <bool kRHA>
-__device__ __forceinline__ uint32_t encode_group_fp32(const uint32_t (&xb)[4], const float (&t)[4], uint32_t p16,
-                                                      uint32_t e8, uint32_t& e16) {
-  e16 = p16 >= 0x40000000u + (e8 << 23);                          // >= 2.0 * 2^e8
-  const float mul = __uint_as_float((129u - (e8 + e16)) << 23);   // 4 * 2^-(e8+e16)
-  uint32_t half = 0;
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    uint32_t m;
-    if (!kRHA) {
-      // t * mul is exact (power of two); adding 1.5 * 2^23 rounds it to an integer, nearest-even, in
-      // the low mantissa bits; the integer minimum clamps to 7 and also catches Inf
-      m = min(__float_as_uint(__fmaf_rn(t[e], mul, 12582912.0f)), 0x4B400007u) & 7u;
-    } else {
-      const float q = fminf(__fmul_rn(t[e], mul), 8.0f);
-      const float fl = truncf(q);
-      m = min(static_cast<uint32_t>(fl) + ((q - fl) >= 0.5f ? 1u : 0u), 7u);
-    }
-    half += (m | ((xb[e] >> 28) & 8u)) << (4 * e);
-  }
-  return half;
-}
-
 // 4 lanes per unit.  Lane l loads the level-3 groups l, l + 4, l + 8, l + 12 (4 elements each: 16-byte chunks
 // of an FP32 unit, 8-byte chunks of an FP16 unit); lanes 2w', 2w'+1 together hold the level-2
 // groups w' + 2c (c = 0..3).  A warp covers 8 units per pass.
 constexpr int kUnrollFp32 = 2;
-
-// Four consecutive source elements (one level-3 group) as FP32 bit patterns.  FP16 elements are widened,
-// which is exact, so an FP16 tensor encodes like the FP32 tensor of the same values.
-__device__ __forceinline__ uint4 load_group_fp32(const float* p) { return ld_stream(reinterpret_cast<const uint4*>(p)); }
-__device__ __forceinline__ uint4 load_group_fp32(const __half* p) {
-  uint2 h;
-  asm volatile("ld.global.cs.v2.u32 {%0,%1}, [%2];" : "=r"(h.x), "=r"(h.y) : "l"(p));
-  const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&h.x));
-  const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&h.y));
-  return make_uint4(__float_as_uint(lo.x), __float_as_uint(lo.y), __float_as_uint(hi.x), __float_as_uint(hi.y));
-}
 
 template <bool kRHA, bool kContig, typename Src>
 __global__ void __launch_bounds__(kThreads)
@@ -218,54 +174,8 @@ quantize_fp32_kernel(const Src* __restrict__ src, int64_t n_units, int64_t upr, 
 #pragma unroll
   for (int i = 0; i < kUnrollFp32; ++i) {
     const int64_t u = first + 8 * i;
-    uint32_t xb[4][4], ab[4][4];
-    uint32_t vm = 0u;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      xb[c][0] = v[i][c].x; xb[c][1] = v[i][c].y; xb[c][2] = v[i][c].z; xb[c][3] = v[i][c].w;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) { ab[c][e] = xb[c][e] & 0x7FFFFFFFu; vm = max(vm, ab[c][e]); }
-    }
-    vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 1));
-    vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 2));
-    const bool unit_nan = vm > 0x7F800000u;
-
-    const float sf = __fmul_rn(__uint_as_float(vm), __uint_as_float(0x3E124925u));   // (1/7)_FP32
-    const uint32_t byte = e6m2_from_bits<23, kRHA>(__float_as_uint(sf));
-    const uint32_t M = byte & 3u;
-    // nearest FP32 of 1, 0.8, 2/3, 4/7
-    const uint32_t lut = M == 0 ? 0x3F800000u : M == 1 ? 0x3F4CCCCDu : M == 2 ? 0x3F2AAAABu : 0x3F124925u;
-    const float rec = __uint_as_float(lut + (48u << 23) - ((byte >> 2) << 23));
-
-    uint32_t half[4], meta = 0u;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      float t[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) t[e] = __fmul_rn(__uint_as_float(ab[c][e]), rec);
-      const uint32_t p16 = max(max(__float_as_uint(t[0]), __float_as_uint(t[1])),
-                               max(__float_as_uint(t[2]), __float_as_uint(t[3])));
-      // level-2 peak: this lane's level-3 group and its neighbour's
-      const uint32_t e8 = max(p16, __shfl_xor_sync(0xFFFFFFFFu, p16, 1)) >= 0x40800000u;    // >= 4.0
-      uint32_t e16;
-      half[c] = encode_group_fp32<kRHA>(xb[c], t, p16, e8, e16);
-      // level-3 group l + 4c -> E1_16 bit 16 + l + 4c; its level-2 group (l >> 1) + 2c -> E1_8 bit, set by the even lane
-      meta |= e16 << (16 + l + 4 * c);
-      if ((l & 1) == 0) meta |= e8 << (8 + (l >> 1) + 2 * c);
-    }
-    // even lane: word (l >> 1) + 2c = its four nibbles | the odd neighbour's << 16
-    const uint32_t mine01 = half[0] | (half[1] << 16), mine23 = half[2] | (half[3] << 16);
-    const uint32_t other01 = __shfl_xor_sync(0xFFFFFFFFu, mine01, 1), other23 = __shfl_xor_sync(0xFFFFFFFFu, mine23, 1);
-    uint32_t codes[4] = {(mine01 & 0xFFFFu) | (other01 << 16), (mine01 >> 16) | (other01 & 0xFFFF0000u),
-                         (mine23 & 0xFFFFu) | (other23 << 16), (mine23 >> 16) | (other23 & 0xFFFF0000u)};
-    meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 1);
-    meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 2);
-    meta |= byte;
-    if (unit_nan) {
-      meta = 0xFFu;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) codes[c] = 0u;
-    }
+    uint32_t codes[4], meta;
+    encode_unit_fp32_quad<kRHA>(v[i], l, codes, meta);
 
     if (u < n_units) {
       uint32_t* out = dst + u * kUnitWords;
