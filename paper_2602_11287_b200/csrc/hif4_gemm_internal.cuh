@@ -23,7 +23,7 @@ hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, i
                             void* workspace, size_t workspace_bytes, cudaStream_t st);
 // Weight-streaming path for M <= kGemvMaxM tokens (mma.sync on register-decoded weights): needs
 // K % 256 == 0, 16-byte aligned B and a workspace of gemv_workspace_bytes (the decoded tokens).
-constexpr int64_t kGemvMaxM = 16;
+constexpr int64_t kGemvMaxM = 32;
 bool gemv_supported(const void* A, const void* B, int64_t M, int64_t N, int64_t K);
 size_t gemv_workspace_bytes(int64_t M, int64_t K);
 hif4_status launch_gemv(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,

@@ -437,14 +437,16 @@ hif4_status launch_gemv_t(const void* B, int64_t upr, GemvParams p, cudaStream_t
 
 }  // namespace
 
+// Token rows are padded to whole MMA n-tiles of 8: one, two or four of them.
+static int64_t gemv_m_pad(int64_t M) { return M <= 8 ? 8 : M <= 16 ? 16 : 32; }
+
 bool gemv_supported(const void* A, const void* B, int64_t M, int64_t N, int64_t K) {
   return M >= 1 && M <= kGemvMaxM && gemm_tc_supported(B, B, N, N, N, K) && (reinterpret_cast<uintptr_t>(A) & 3u) == 0;
 }
 
 size_t gemv_workspace_bytes(int64_t M, int64_t K) {
   if (M < 1 || M > kGemvMaxM || K <= 0 || K % 256 != 0) return 0;
-  const int64_t m_pad = M <= 8 ? 8 : 16;
-  return static_cast<size_t>(m_pad * K * 2);
+  return static_cast<size_t>(gemv_m_pad(M) * K * 2);
 }
 
 namespace {
@@ -466,6 +468,7 @@ hif4_status launch_gemv_stream(const void* B, const GemvParams& p, int m_pad, in
   const int64_t rounds = ceil_div64(p.num_blocks, sms * kMaxBlocks);
   const int64_t grid = p.num_blocks < sms * rounds ? p.num_blocks : sms * rounds;
   const bool many = ceil_div64(p.num_blocks, grid) >= 9;
+  if (m_pad == 32) return launch_gemv_t<4, kGemvWarpsFew>(B, upr, p, st);      // four token tiles: registers for 24 warps only
   if (m_pad == 8) return many ? launch_gemv_t<1, kGemvWarpsMany>(B, upr, p, st) : launch_gemv_t<1, kGemvWarpsFew>(B, upr, p, st);
   return many ? launch_gemv_t<2, kGemvWarpsMany>(B, upr, p, st) : launch_gemv_t<2, kGemvWarpsFew>(B, upr, p, st);
 }
@@ -477,7 +480,7 @@ hif4_status launch_gemv(const void* A, const void* B, float* C, int64_t M, int64
   p.A = static_cast<const uint32_t*>(A);
   if (!gemv_params(p, C, M, N, K, ldc, workspace)) return HIF4_ERR_SHAPE;
   if (!p.error_word) return HIF4_ERR_CUDA;
-  const int m_pad = M <= 8 ? 8 : 16;
+  const int m_pad = static_cast<int>(gemv_m_pad(M));
   const int64_t upr = K / kUnitElems;
   const int64_t prep = static_cast<int64_t>(m_pad) * upr;
   gemv_prepare_tokens_kernel<<<static_cast<unsigned>(ceil_div64(prep, 128)), 128, 0, st>>>(p.A, p.M, m_pad, upr, p.tokens);
@@ -497,7 +500,7 @@ hif4_status launch_gemv_linear(const void* X, hif4_dtype dt, int64_t ld_x, int r
   GemvParams p{};
   if (!gemv_params(p, C, M, N, K, ldc, workspace)) return HIF4_ERR_SHAPE;
   if (!p.error_word) return HIF4_ERR_CUDA;
-  const int m_pad = M <= 8 ? 8 : 16;
+  const int m_pad = static_cast<int>(gemv_m_pad(M));
   const int64_t upr = K / kUnitElems;
   const int lanes = dt == HIF4_BF16 ? 2 : 4;             // lanes per unit of the encoder
   const unsigned blocks = static_cast<unsigned>(ceil_div64(lanes * static_cast<int64_t>(m_pad) * upr, 128));

@@ -56,9 +56,9 @@ def test_small_and_ragged_shapes(hif4, M, N, K):
     check_full(hif4, hif4.hif4_quantize(a), hif4.hif4_quantize(b), f"{M}x{N}x{K}")
 
 
-@pytest.mark.parametrize("M,N,K", [(17, 300, 256), (40, 257, 768), (100, 1000, 1024), (128, 512, 2048), (65, 31, 256)])
+@pytest.mark.parametrize("M,N,K", [(33, 300, 256), (40, 257, 768), (100, 1000, 1024), (128, 512, 2048), (65, 31, 256)])
 def test_few_rows_default_path(hif4, M, N, K):
-    """17 <= M <= 128 with K % 256 == 0 goes to the CTA-pair kernel with swapped operands."""
+    """33 <= M <= 128 with K % 256 == 0 goes to the CTA-pair kernel with swapped operands."""
     g = torch.Generator(device="cuda"); g.manual_seed(M * 13 + N)
     a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
     b = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
@@ -322,13 +322,14 @@ def gemv_path(hif4):
 
 @pytest.mark.parametrize("M,N,K", [(1, 1, 256), (1, 64, 256), (2, 33, 512), (7, 200, 1024), (8, 4096, 256), (9, 130, 768),
                                    (16, 1000, 2304), (16, 64, 4096), (5, 9475, 256), (3, 31, 5120), (12, 77, 14336),
-                                   (1, 40003, 256), (16, 2376, 1024), (10, 1192, 512), (4, 19000, 256)])
+                                   (1, 40003, 256), (16, 2376, 1024), (10, 1192, 512), (4, 19000, 256),
+                                   (17, 300, 256), (32, 1000, 1024), (25, 4200, 512), (31, 77, 4096), (20, 14336, 256)])
 def test_weight_streaming_kernel_full_compare(gemv_path, M, N, K):
     hif4 = gemv_path
     g = torch.Generator(device="cuda"); g.manual_seed(M * 11 + N)
     a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
     b = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
-    assert hif4.hif4_gemm_workspace(M, N, K) == (8 if M <= 8 else 16) * K * 2
+    assert hif4.hif4_gemm_workspace(M, N, K) == (8 if M <= 8 else 16 if M <= 16 else 32) * K * 2
     before = hif4.launch_count()
     out = torch.full((M + 2, N + 3), -5.0, dtype=torch.float32, device="cuda")
     C = check_full(hif4, a, b, f"gemv {M}x{N}x{K}", out=out[1:M + 1, 1:N + 1])
