@@ -109,8 +109,8 @@ hif4_status hif4_dequantize(const void* src_units, int64_t rows, int64_t cols, v
                             hif4_dtype dt, int64_t ld_dst, void* stream);
 
 /* Workspace (device scratch) that hif4_gemm needs for this shape on the current device; may be 0.
- * For M <= 16 it holds the decoded activation rows (2 * K * 8 or 16 bytes); for large M a few KB of
- * completion words when the last round of the tile schedule is split along K.  Host-only.  */
+ * For M <= 32 it holds the decoded activation rows (2 * K * 8, 16 or 32 bytes); for larger M a few KB of
+ * completion words when tiles are split along K.  Host-only.  */
 hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size_t* bytes);
 
 /* hif4_gemm -- C = A * B^T with A, B in HiF4 and FP32 accumulation: C[i][j] is the sum over the

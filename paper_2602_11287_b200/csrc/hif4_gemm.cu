@@ -27,6 +27,10 @@ extern "C" hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size
   if (!bytes) return HIF4_ERR_NULL;
   if (M < 0 || N < 0 || K < 0 || K % kUnitElems != 0) return HIF4_ERR_SHAPE;
   *bytes = gemv_workspace_bytes(M, K);       // decoded tokens of the weight-streaming path (M <= 16)
+  if (g_gemm_path == 0 && M > kGemvMaxM && M < kPairMinM) {
+    const size_t few_bytes = gemm_tc2_swapped_workspace_bytes(M, N, K);  // completion words of the K slices
+    if (few_bytes > *bytes) *bytes = few_bytes;
+  }
   if (g_gemm_path == 3 || (g_gemm_path == 0 && M >= kPairMinM)) {
     const size_t pair_bytes = gemm_tc2_workspace_bytes(M, N, K);     // completion words of a K-sliced last round
     if (pair_bytes > *bytes) *bytes = pair_bytes;
@@ -63,8 +67,10 @@ extern "C" hif4_status hif4_gemm(const void* A_units, const void* B_units, float
     return launch_gemm_tc2(A_units, B_units, C, M, N, K, ldc, workspace, workspace_bytes, st);
   }
   // few rows: the pair kernel with the operands swapped pads them to 32 instead of 128
-  if (tc_ok && g_gemm_path == 0 && M > kGemvMaxM && M < kPairMinM && gemm_tc2_supported(A_units, B_units, M, N, K))
-    return launch_gemm_tc2_swapped(A_units, B_units, C, M, N, K, ldc, st);
+  if (tc_ok && g_gemm_path == 0 && M > kGemvMaxM && M < kPairMinM && gemm_tc2_supported(A_units, B_units, M, N, K)) {
+    if (workspace && !aligned(workspace, 256)) return HIF4_ERR_ALIGN;
+    return launch_gemm_tc2_swapped(A_units, B_units, C, M, N, K, ldc, workspace, workspace_bytes, st);
+  }
   if (tc_ok && (g_gemm_path >= 2 || M > kGemvMaxM)) return launch_gemm_tc(A_units, B_units, C, M, N, K, ldc, st);
   return launch_gemm_simt(A_units, B_units, C, M, N, K, ldc, st);
 }

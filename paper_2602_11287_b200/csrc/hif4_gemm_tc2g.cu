@@ -49,6 +49,11 @@ struct GroupedParams {
   int max_entries;
   const TokTile* table;     // nullptr: one dense problem of dense_rows token rows (a single tile)
   int dense_rows;
+  // Dense problems with fewer weight tiles than CTA pairs: every tile is cut into `slices` K ranges on pairs of
+  // their own.  Slice 0 stores its part of C, slice s > 0 adds to it after the same epilogue warp of slice s - 1
+  // is done with the same columns, so every element is summed in slice order.
+  int slices;               // 1: not split (always 1 with a table)
+  unsigned int* flags;      // [n_wtiles][slices][8]: "this epilogue warp of this slice is done" (zero at launch)
   unsigned int* error_word;
   DecodeMul mul;
 };
@@ -79,15 +84,27 @@ __global__ void build_toktile_table_kernel(const int64_t* __restrict__ offsets, 
   }
 }
 
-struct Unit { int tok0; int tok_end; int T; int w_row0; int n0; bool valid; };
+struct Unit { int tok0; int tok_end; int T; int w_row0; int n0; int kc0; int kc1; int wt; int slice; bool valid; };
 __device__ __forceinline__ Unit unit_of(const GroupedParams& p, int u) {
-  const int e = u / p.n_wtiles, wt = u - e * p.n_wtiles;
-  const TokTile t = p.table ? p.table[e] : TokTile{0, p.dense_rows, 0, (p.dense_rows + 31) & ~31};
   Unit r;
+  if (p.table == nullptr) {                 // dense: unit = (K slice, weight tile)
+    r.slice = u / p.n_wtiles; r.wt = u - r.slice * p.n_wtiles;
+    r.tok0 = 0; r.tok_end = p.dense_rows; r.T = (p.dense_rows + 31) & ~31;
+    r.valid = true;
+    r.n0 = r.wt * 256;
+    r.w_row0 = r.n0;
+    r.kc0 = static_cast<int>(static_cast<int64_t>(r.slice) * p.num_kc / p.slices);
+    r.kc1 = static_cast<int>(static_cast<int64_t>(r.slice + 1) * p.num_kc / p.slices);
+    return r;
+  }
+  const int e = u / p.n_wtiles;
+  r.wt = u - e * p.n_wtiles; r.slice = 0;
+  const TokTile t = p.table[e];
   r.valid = t.group >= 0;
   r.tok0 = t.tok0; r.tok_end = t.tok_end; r.T = t.T;
-  r.n0 = wt * 256;
+  r.n0 = r.wt * 256;
   r.w_row0 = static_cast<int>(t.group * p.N) + r.n0;
+  r.kc0 = 0; r.kc1 = p.num_kc;
   return r;
 }
 
@@ -106,6 +123,24 @@ __device__ __forceinline__ bool decode_two_units_g(const uint32_t (&W)[18], bool
     if ((threadIdx.x & 31) == 0) mbar_arrive_cluster(dec_full0_leader + 8 * u);
   }
   return true;
+}
+
+// Bounded wait until a word in global memory, written by another CTA after a __threadfence(), has reached `want`.
+__device__ __noinline__ bool wait_word(const unsigned int* word, unsigned int want, volatile uint32_t* abort_flag) {
+  const uint64_t t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(word) : "memory");
+    if (v >= want) return true;
+    __nanosleep(32);
+    if ((it & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > kWaitBudgetNs) {
+        *abort_flag = 1u;
+        return false;
+      }
+    }
+  }
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
@@ -128,7 +163,7 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-  const int total_units = p.max_entries * p.n_wtiles;
+  const int total_units = p.max_entries * p.n_wtiles * p.slices;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kRawStages; ++s) {
@@ -166,7 +201,7 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
       for (int u = pair; u < total_units && ok; u += num_pairs) {
         const Unit un = unit_of(p, u);
         if (!un.valid) continue;
-        for (int kc = 0; kc < p.num_kc; ++kc, ++n) {
+        for (int kc = un.kc0; kc < un.kc1; ++kc, ++n) {
           const uint32_t s = n & 1u, ph = (n >> 1) & 1u;
           if (!(ok = mbar_wait(raw_empty + 8 * s, ph ^ 1u, abort_flag, 128))) break;
           mbar_expect_tx(raw_full + 8 * s, kRawStageBytes);
@@ -190,7 +225,7 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * kMaxTok;
         const uint32_t idesc = kInstrDescM256 | (static_cast<uint32_t>(un.T >> 3) << 17);
-        for (int kc = 0; kc < p.num_kc && ok; ++kc, ++n) {
+        for (int kc = un.kc0; kc < un.kc1 && ok; ++kc, ++n) {
           // stages 0 and 2 are filled first (see the dense pair kernel): consume 0, 2, 1, 3
 #pragma unroll
           for (int i = 0; i < kDecStages; ++i) {
@@ -201,7 +236,7 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
             const uint64_t bdesc = make_desc(dec_base + st * kDecStageBytes + kDecHalfBytes);  // tokens: N side
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-              tc2_mma(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kc | i | kk) != 0 ? 1u : 0u);
+              tc2_mma(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, ((kc - un.kc0) | i | kk) != 0 ? 1u : 0u);
             tc2_commit_both(dec_empty + 8 * st);
           }
         }
@@ -224,6 +259,10 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
       const int64_t col = static_cast<int64_t>(un.n0) + rank * kWRows + q * 32 + lane;      // column of C = weight row
       const bool col_ok = col < p.N;
       const int chunks = un.T >> 4;
+      // K-sliced dense tile: slices after the first add to what the previous slice has left in C
+      const bool adds = un.slice > 0;
+      unsigned int* my_flag = p.slices > 1 ? p.flags + (static_cast<size_t>(un.wt) * p.slices + un.slice) * 8 + rank * 4 + q : nullptr;
+      if (adds && !__all_sync(0xFFFFFFFFu, wait_word(my_flag - 8, 1u, abort_flag))) break;
 #pragma unroll 1
       for (int c = 0; c < chunks; ++c) {
         uint32_t r[16];
@@ -238,7 +277,16 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
         float* cp = p.C + static_cast<int64_t>(tok) * p.ldc + col;
 #pragma unroll
         for (int v = 0; v < 16; ++v)
-          if (col_ok && tok + v < un.tok_end) cp[static_cast<int64_t>(v) * p.ldc] = __uint_as_float(r[v]);
+          if (col_ok && tok + v < un.tok_end) {
+            float* dst = cp + static_cast<int64_t>(v) * p.ldc;
+            if (adds) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst), "f"(__uint_as_float(r[v])) : "memory");
+            else *dst = __uint_as_float(r[v]);
+          }
+      }
+      if (p.slices > 1 && un.slice + 1 < p.slices) {      // the next slice may add to these columns now
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(my_flag), "r"(1u) : "memory");
       }
       ++ucount;
     }
@@ -261,7 +309,7 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
       const Unit un = unit_of(p, u);
       if (!un.valid) continue;
       const bool active = row < 128 || (row - 128) < (un.T >> 1);
-      for (int kc = 0; kc < p.num_kc && ok; ++kc, ++n) {
+      for (int kc = un.kc0; kc < un.kc1 && ok; ++kc, ++n) {
         const uint32_t s = n & 1u, ph = (n >> 1) & 1u;
         if (!(ok = __all_sync(0xFFFFFFFFu, mbar_wait(raw_full + 8 * s, ph, abort_flag)))) break;
         uint32_t L[20];
@@ -309,7 +357,8 @@ hif4_status launch_swapped(const void* A, const void* B, int64_t a_rows, int64_t
   p.error_word = device_error_word();
   if (!p.error_word) return HIF4_ERR_CUDA;
   p.mul = make_decode_mul();
-  const int64_t units = static_cast<int64_t>(p.max_entries) * p.n_wtiles;
+  if (p.slices < 1) p.slices = 1;
+  const int64_t units = static_cast<int64_t>(p.max_entries) * p.n_wtiles * p.slices;
   if (units > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
   const int pairs = static_cast<int>(units < sm_count() / 2 ? units : sm_count() / 2);
   gemm_tc2g_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tmTok, tmW, p);
@@ -319,14 +368,42 @@ hif4_status launch_swapped(const void* A, const void* B, int64_t a_rows, int64_t
 
 }  // namespace
 
+// K slices of a dense problem with few rows.  All slices of all weight tiles must be resident at once (they wait
+// for one another), and a slice starts its epilogue when the one before it has finished its own, which costs
+// about the time of 3.5 K = 256 chunks per extra slice: take the count with the shortest critical path, at most 4.
+static int swapped_slices(int64_t N, int64_t K) {
+  const int64_t tiles = ceil_div64(N, 256), pairs = sm_count() / 2, chunks = K / 256;
+  int64_t s_max = tiles > 0 ? pairs / tiles : 1;
+  if (s_max > 4) s_max = 4;
+  int64_t best = 1, best_cost = 2 * chunks;
+  for (int64_t s = 2; s <= s_max; ++s) {
+    const int64_t cost = 2 * ceil_div64(chunks, s) + 7 * (s - 1);       // in half chunks
+    if (cost < best_cost) { best = s; best_cost = cost; }
+  }
+  return static_cast<int>(best);
+}
+
+size_t gemm_tc2_swapped_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  if (M <= 0 || N <= 0 || K <= 0 || K % 256 != 0) return 0;
+  const int s = swapped_slices(N, K);
+  return s > 1 ? static_cast<size_t>((ceil_div64(N, 256) * s * 8 * sizeof(unsigned int) + 255) / 256 * 256) : 0;
+}
+
 // Dense problem with few rows (M <= 128): the same kernel with a single token tile.
 hif4_status launch_gemm_tc2_swapped(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K,
-                                    int64_t ldc, cudaStream_t st) {
+                                    int64_t ldc, void* workspace, size_t workspace_bytes, cudaStream_t st) {
   GroupedParams p{};
   p.C = C; p.ldc = ldc; p.N = N;
   p.max_entries = 1;
   p.table = nullptr;
   p.dense_rows = static_cast<int>(M);
+  p.slices = swapped_slices(N, K);
+  if (p.slices > 1) {
+    const size_t need = gemm_tc2_swapped_workspace_bytes(M, N, K);
+    if (!workspace || workspace_bytes < need) return HIF4_ERR_WORKSPACE;
+    p.flags = static_cast<unsigned int*>(workspace);
+    if (cudaMemsetAsync(p.flags, 0, need, st) != cudaSuccess) return HIF4_ERR_CUDA;
+  }
   return launch_swapped(A, B, M, N, p, K, st);
 }
 

@@ -56,9 +56,11 @@ def test_small_and_ragged_shapes(hif4, M, N, K):
     check_full(hif4, hif4.hif4_quantize(a), hif4.hif4_quantize(b), f"{M}x{N}x{K}")
 
 
-@pytest.mark.parametrize("M,N,K", [(33, 300, 256), (40, 257, 768), (100, 1000, 1024), (128, 512, 2048), (65, 31, 256)])
+@pytest.mark.parametrize("M,N,K", [(33, 300, 256), (40, 257, 768), (100, 1000, 1024), (128, 512, 2048), (65, 31, 256),
+                                   (40, 500, 4096), (100, 1000, 2048), (128, 4096, 4096), (64, 2100, 3072)])
 def test_few_rows_default_path(hif4, M, N, K):
-    """33 <= M <= 128 with K % 256 == 0 goes to the CTA-pair kernel with swapped operands."""
+    """33 <= M <= 128 with K % 256 == 0 goes to the CTA-pair kernel with swapped operands; with few weight tiles and a
+    long K every tile is cut into up to four K slices that are added in slice order (the last four shapes)."""
     g = torch.Generator(device="cuda"); g.manual_seed(M * 13 + N)
     a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
     b = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
