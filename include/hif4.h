@@ -200,7 +200,7 @@ const char* hif4_status_string(hif4_status s);
 /* Diagnostic: 0 = choose the GEMM kernel by shape (default), 1 = CUDA-core kernel only, 2 = the
  * single-CTA tensor-core (tcgen05) kernel whenever it is legal (K % 256 == 0, 16-byte aligned
  * operands), even for small M, 3 = the CTA-pair tensor-core kernel (256 x 256 tiles) whenever it is
- * legal, 4 = the weight-streaming kernel whenever it is legal (M <= 16).  Process-wide, not
+ * legal, 4 = the weight-streaming kernel whenever it is legal (M <= 32).  Process-wide, not
  * thread-safe; meant for tests and benchmarks.  */
 hif4_status hif4_set_gemm_path(int path);
 

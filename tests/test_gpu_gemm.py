@@ -447,9 +447,10 @@ def test_linear_is_quantize_then_gemm(hif4, M, N, K, dtype):
 
 @pytest.mark.parametrize("mode", [0, 1])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32, torch.float16])
-@pytest.mark.parametrize("M,N,K", [(1, 4096, 4096), (16, 1000, 1024), (7, 260, 256), (9, 64, 2304), (16, 14336, 4096)])
+@pytest.mark.parametrize("M,N,K", [(1, 4096, 4096), (16, 1000, 1024), (7, 260, 256), (9, 64, 2304), (16, 14336, 4096),
+                                   (24, 520, 1024), (32, 64, 256)])
 def test_linear_with_few_rows_quantizes_inside_the_token_preparation(hif4, M, N, K, dtype, mode):
-    """M <= 16 rows of activations: hif4_linear runs two kernels (quantize-and-decode of the tokens, weight
+    """M <= 32 rows of activations: hif4_linear runs two kernels (quantize-and-decode of the tokens, weight
     streaming) instead of three and gives exactly the bits of hif4_quantize followed by hif4_gemm -- on a strided
     source with spikes, a NaN and an Inf, for every source type and both rounding modes."""
     g = torch.Generator(device="cuda"); g.manual_seed(M * 3 + N + K + mode)
