@@ -7,7 +7,9 @@ quantized to HiF4 (Algorithm 1) and multiplied with the pre-quantized HiF4 weigh
 accumulation).  All inputs are seeded synthetic tensors (Student-t activations with outlier
 channels, Gaussian weights); the model name only lends the layer shapes.
 
-Prints ONE JSON line (see README for the keys).  `--impl reference` times the CPU oracle
+Prints ONE JSON line: metric, value (whole-job TFLOP/s with inputs resident), ms_per_step, gpu_launches, clocks,
+roofline (the prefill GEMM kernel against the measured BF16 peak), per_shape, roofline_quantize, reference_points,
+e2e (through host buffers) and cpu_baseline.  `--impl reference` times the CPU oracle
 on a bounded sample of the same workload instead.
 """
 from __future__ import annotations
