@@ -66,15 +66,23 @@ struct Gemm2Params {
   int total_tiles;
   unsigned int* error_word;
   int tma_store;        // 1: C goes out through the tensor map tmC, 0: per-thread stores
-  // Tail of the tile schedule: every pair computes `full_rounds` whole tiles; the `tail_tiles` tiles that
-  // are left (fewer than there are pairs) are cut into `slices` K ranges each, so that the last round
+  // Tile schedule: every pair computes `full_rounds` whole tiles.  Fewer tiles than pairs (full_rounds == 0): the
+  // `tail_tiles` tiles are cut into `slices` K ranges each, on pairs of their own, so that the single round
   // keeps tail_tiles * slices pairs busy instead of tail_tiles.  Slice 0 of a tile stores its part to C,
   // slice s > 0 adds its part with TMA reduce-add stores once slice s - 1 has finished the same rows
   // (warp to warp: an epilogue warp owns 32 rows of the tile), so every element is summed in slice order.
   int full_rounds;
   int tail_tiles;
   int slices;               // 1: tail tiles are not split
-  unsigned int* flags;      // [tail_tiles][slices][8]: "this epilogue warp's rows of this slice are in C" (zero at launch)
+  // Balanced last rounds (sk_tiles > 0; then tail_tiles is 0 and slices is 2): after `full_rounds` whole tiles per
+  // pair, the K = 256 chunks of the remaining `sk_tiles` tiles (between one and two per pair, starting at tile
+  // `sk_tile0`), laid end to end, are dealt out in equal contiguous runs.  A run begins with the last chunks of a
+  // tile whose first chunks end the previous pair's run: the pair that has the end of a tile computes it first and
+  // stores it (slice 0, flag row = its own index), the pair that has the beginning computes it last and adds
+  // (slice 1), so the addition hardly ever waits.
+  int sk_tiles;
+  int sk_tile0;
+  unsigned int* flags;      // [tail_tiles or pairs + 1][slices][8]: "this epilogue warp's rows of this slice are in C" (zero at launch)
   DecodeMul mul;
 };
 
@@ -86,7 +94,18 @@ struct WorkItem {
   int tail;             // index among the tail tiles, -1 for a whole tile
   int slice;            // K slice of a tail tile
 };
-__device__ __forceinline__ int num_work_items(const Gemm2Params& p, int pair) {
+// First and last chunk (exclusive) of a pair's run in the balanced rounds, in chunks of the sk_tiles tiles laid end to end.
+__device__ __forceinline__ void balanced_run(const Gemm2Params& p, int pair, int num_pairs, int64_t& c0, int64_t& c1) {
+  const int64_t total = static_cast<int64_t>(p.sk_tiles) * p.num_kc;
+  c0 = total * pair / num_pairs;
+  c1 = total * (pair + 1) / num_pairs;
+}
+__device__ __forceinline__ int num_work_items(const Gemm2Params& p, int pair, int num_pairs) {
+  if (p.sk_tiles > 0) {
+    int64_t c0, c1;
+    balanced_run(p, pair, num_pairs, c0, c1);
+    return p.full_rounds + static_cast<int>((c1 - 1) / p.num_kc - c0 / p.num_kc) + 1;
+  }
   return p.full_rounds + (pair < p.tail_tiles * p.slices ? 1 : 0);
 }
 __device__ __forceinline__ WorkItem work_item(const Gemm2Params& p, int pair, int num_pairs, int i) {
@@ -95,6 +114,17 @@ __device__ __forceinline__ WorkItem work_item(const Gemm2Params& p, int pair, in
   if (i < p.full_rounds) {
     t = i * num_pairs + pair;
     w.kc0 = 0; w.kc1 = p.num_kc; w.tail = -1; w.slice = 0;
+  } else if (p.sk_tiles > 0) {
+    int64_t c0, c1;
+    balanced_run(p, pair, num_pairs, c0, c1);
+    const int64_t tr = c0 / p.num_kc + (i - p.full_rounds);
+    const int64_t first = tr * p.num_kc;
+    w.kc0 = c0 > first ? static_cast<int>(c0 - first) : 0;
+    w.kc1 = c1 < first + p.num_kc ? static_cast<int>(c1 - first) : p.num_kc;
+    t = p.sk_tile0 + static_cast<int>(tr);
+    if (w.kc0 > 0) { w.tail = pair; w.slice = 0; }                       // end of a tile: computed first, stored
+    else if (w.kc1 < p.num_kc) { w.tail = pair + 1; w.slice = 1; }       // beginning of a tile: computed last, added
+    else { w.tail = -1; w.slice = 0; }
   } else {
     w.tail = pair % p.tail_tiles;
     w.slice = pair / p.tail_tiles;
@@ -168,7 +198,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-  const int n_items = num_work_items(p, pair);
+  const int n_items = num_work_items(p, pair, num_pairs);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kRawStages; ++s) {
@@ -416,7 +446,7 @@ bool make_c_map(CUtensorMap* map, float* C, int64_t M, int64_t N, int64_t ldc) {
 
 // Tile schedule of the dense pair kernel for this shape on this device (see Gemm2Params).
 struct Tc2Plan {
-  int pairs, full_rounds, tail_tiles, slices;
+  int pairs, full_rounds, tail_tiles, slices, sk_tiles, sk_tile0;
   size_t flag_bytes, bytes;          // workspace: the slices' completion words
 };
 static Tc2Plan tc2_plan(int64_t M, int64_t N, int64_t K) {
@@ -445,7 +475,18 @@ static Tc2Plan tc2_plan(int64_t M, int64_t N, int64_t K) {
     }
     pl.slices = static_cast<int>(best);
   }
-  if (pl.slices > 1) {
+  if (pl.full_rounds >= 1 && pl.tail_tiles > 0) {
+    // Several rounds and a partial one: the last whole round and the partial one are balanced chunk by chunk
+    // instead (every pair then works tail_tiles / pairs of a tile longer than the whole rounds take, which is never
+    // more than the K slices of the partial round alone would cost).
+    pl.full_rounds -= 1;
+    pl.sk_tile0 = pl.full_rounds * pl.pairs;
+    pl.sk_tiles = pl.pairs + pl.tail_tiles;
+    pl.tail_tiles = 0;
+    pl.slices = 2;
+    pl.flag_bytes = (static_cast<size_t>(pl.pairs + 1) * 2 * 8 * sizeof(unsigned int) + 255) / 256 * 256;
+    pl.bytes = pl.flag_bytes;
+  } else if (pl.slices > 1) {
     pl.flag_bytes = (static_cast<size_t>(pl.tail_tiles) * pl.slices * 8 * sizeof(unsigned int) + 255) / 256 * 256;
     pl.bytes = pl.flag_bytes;
   }
@@ -485,12 +526,19 @@ hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, i
   p.full_rounds = pl.full_rounds;
   p.tail_tiles = pl.tail_tiles;
   p.slices = p.tma_store ? pl.slices : 1;             // the plain-store epilogue cannot add to C
+  p.sk_tiles = pl.sk_tiles;
+  p.sk_tile0 = pl.sk_tile0;
+  if (p.sk_tiles > 0 && !p.tma_store) {               // back to whole tiles: full rounds and an unsliced partial one
+    p.full_rounds += 1;
+    p.tail_tiles = p.sk_tiles - pl.pairs;
+    p.sk_tiles = 0;
+  }
   if (p.slices > 1) {
     if (!workspace || workspace_bytes < pl.bytes) return HIF4_ERR_WORKSPACE;
     p.flags = static_cast<unsigned int*>(workspace);
     if (cudaMemsetAsync(p.flags, 0, pl.flag_bytes, st) != cudaSuccess) return HIF4_ERR_CUDA;
   }
-  const int pairs = p.full_rounds == 0 ? p.tail_tiles * p.slices : pl.pairs;      // a single round: one pair per slice
+  const int pairs = p.full_rounds == 0 && p.sk_tiles == 0 ? p.tail_tiles * p.slices : pl.pairs;      // a single round: one pair per slice
   gemm_tc2_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tmA, tmB, tmC, p);
   note_launch();
   return launch_status();

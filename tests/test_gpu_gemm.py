@@ -255,11 +255,12 @@ def test_cta_pair_kernel_few_columns_in_the_last_tile_repeated(hif4):
 
 
 @pytest.mark.parametrize("M,N,K", [(2560, 2048, 16384), (2500, 2000, 8192), (19 * 256, 4 * 256 + 8, 8192), (2560, 2048, 2048),
-                                   (512, 2048, 4096), (300, 1000, 2048)])
+                                   (512, 2048, 4096), (300, 1000, 2048), (2304, 4096, 256), (3000, 3000, 768)])
 def test_cta_pair_kernel_k_sliced_last_round(hif4, M, N, K):
-    """More tiles than CTA pairs with a partial last round: its tiles are cut into K slices that are added to
-    C in slice order (80 tiles on 74 pairs -> 6 tail tiles x 4 or 2 slices; 95 tiles -> 21 tail tiles x 3), and
-    a single round with fewer tiles than half the pairs is sliced the same way (16 tiles x 4, 8 tiles x 2)."""
+    """More tiles than CTA pairs with a partial last round (80 and 95 tiles on 74 pairs): the K chunks of the last
+    whole round and the partial one are dealt out in equal runs, so most of those tiles are computed by two pairs,
+    the end of the tile stored first and the beginning added to it.  A single round with fewer tiles than half the
+    pairs is cut into K slices that are added to C in slice order (16 tiles x 4, 8 tiles x 2)."""
     assert hif4.hif4_gemm_workspace(M, N, K) > 0, "the K-sliced round needs its completion words"
     g = torch.Generator(device="cuda"); g.manual_seed(M + N + K)
     a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
