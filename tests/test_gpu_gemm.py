@@ -255,7 +255,8 @@ def test_cta_pair_kernel_few_columns_in_the_last_tile_repeated(hif4):
 
 
 @pytest.mark.parametrize("M,N,K", [(2560, 2048, 16384), (2500, 2000, 8192), (19 * 256, 4 * 256 + 8, 8192), (2560, 2048, 2048),
-                                   (512, 2048, 4096), (300, 1000, 2048), (2304, 4096, 256), (3000, 3000, 768)])
+                                   (512, 2048, 4096), (300, 1000, 2048), (2304, 4096, 256), (3000, 3000, 768),
+                                   (130, 20000, 1024)])
 def test_cta_pair_kernel_k_sliced_last_round(hif4, M, N, K):
     """More tiles than CTA pairs with a partial last round (80 and 95 tiles on 74 pairs): the K chunks of the last
     whole round and the partial one are dealt out in equal runs, so most of those tiles are computed by two pairs,
