@@ -89,55 +89,68 @@ quantize_bf16_kernel(const uint16_t* __restrict__ src, int64_t n_units, int64_t 
 }
 
 // ----------------------------------------------------------------------------- BF16 quantizer, units down the columns
-// One block converts a tile of 64 rows x 128 columns: the rows are read as they lie (256 bytes each), staged in
-// shared memory, and each pair of lanes then takes two neighbouring columns (one 32-bit word per row) as its
-// two units, lane l again the level-2 groups l, l + 2, l + 4, l + 6 of both.  Same encoder as above, so the units
-// are those of hif4_quantize on the transposed matrix.
+// One 64-thread block converts a tile of 64 rows x 128 columns: the rows are read as they lie (256 bytes each) and
+// staged in shared memory with 16-byte stores; each pair of lanes (l and l + 16 of a warp) then takes four
+// neighbouring columns (one 8-byte load per row) as its four units, lane l again the level-2 groups l, l + 2,
+// l + 4, l + 6 of each.  The 16 lanes of a half warp read 128 consecutive bytes of one row: no bank conflicts,
+// and a quarter of the shared-memory instructions that 4-byte accesses need.  Same encoder as above, so the
+// units are those of hif4_quantize on the transposed matrix.
 constexpr int kTileCols = 128;
-constexpr int kTilePitchWords = kTileCols / 2 + 1;        // 32-bit words per staged row: column reads of consecutive rows hit different banks
+constexpr int kTileThreads = 64;
+constexpr int kTileRowWords = kTileCols / 2;
 
 template <bool kRHA>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kTileThreads)
 quantize_bf16_transposed_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t cols, int64_t ld_src,
                                 uint32_t* __restrict__ dst) {
-  __shared__ uint32_t tile[kUnitElems * kTilePitchWords];
+  __shared__ __align__(16) uint32_t tile[kUnitElems * kTileRowWords];
   // consecutive blocks take consecutive row tiles of the same columns: their units are neighbours in dst
   const int64_t c0 = static_cast<int64_t>(blockIdx.y) * kTileCols;
   const int64_t r0 = static_cast<int64_t>(blockIdx.x) * kUnitElems;
   // 64 rows x 16 chunks of 8 elements; a chunk is inside the matrix or outside as a whole (cols % 8 == 0)
-  for (int i = threadIdx.x; i < kUnitElems * (kTileCols / 8); i += blockDim.x) {
-    const int r = i >> 4, ch = i & 15;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (c0 + 8 * ch < cols) v = ld_stream(reinterpret_cast<const uint4*>(src + (r0 + r) * ld_src + c0 + 8 * ch));
-    uint32_t* t = tile + r * kTilePitchWords + 4 * ch;
-    t[0] = v.x; t[1] = v.y; t[2] = v.z; t[3] = v.w;
+  constexpr int kChunks = kUnitElems * (kTileCols / 8) / kTileThreads;      // 16 per thread
+  uint4 in[kChunks];
+#pragma unroll
+  for (int n = 0; n < kChunks; ++n) {
+    const int i = n * kTileThreads + threadIdx.x, r = i >> 4, ch = i & 15;
+    in[n] = make_uint4(0u, 0u, 0u, 0u);
+    if (c0 + 8 * ch < cols) in[n] = ld_stream(reinterpret_cast<const uint4*>(src + (r0 + r) * ld_src + c0 + 8 * ch));
+  }
+#pragma unroll
+  for (int n = 0; n < kChunks; ++n) {
+    const int i = n * kTileThreads + threadIdx.x;
+    *reinterpret_cast<uint4*>(tile + 4 * i) = in[n];                         // row i / 16, words 4 (i % 16) ..
   }
   __syncthreads();
-  const int l = threadIdx.x & 1, cp = threadIdx.x >> 1;     // columns 2 cp and 2 cp + 1 of the tile
-  uint4 even[4], odd[4];
+  const int lane = threadIdx.x & 31, l = lane >> 4;
+  const int cq = (threadIdx.x >> 5) * 16 + (lane & 15);                      // columns 4 cq .. 4 cq + 3 of the tile
+  uint4 col[4][4];                                                           // [column][group l + 2c]
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
-    const uint32_t* p = tile + (8 * (l + 2 * c)) * kTilePitchWords + cp;           // rows 8 g .. 8 g + 7, both columns
-    uint32_t e[4], o[4];
+    const uint32_t* p = tile + (8 * (l + 2 * c)) * kTileRowWords + 2 * cq;   // rows 8 g .. 8 g + 7, four columns
+    uint32_t e[4][4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const uint32_t a = p[(2 * k) * kTilePitchWords], b2 = p[(2 * k + 1) * kTilePitchWords];
-      e[k] = prmt(a, b2, 0x5410u);                          // low halves: the even column of rows 2k, 2k + 1
-      o[k] = prmt(a, b2, 0x7632u);                          // high halves: the odd column
+      const uint2 a = *reinterpret_cast<const uint2*>(p + (2 * k) * kTileRowWords);
+      const uint2 b2 = *reinterpret_cast<const uint2*>(p + (2 * k + 1) * kTileRowWords);
+      e[0][k] = prmt(a.x, b2.x, 0x5410u);                     // low halves: column 0 of rows 2k, 2k + 1
+      e[1][k] = prmt(a.x, b2.x, 0x7632u);                     // high halves: column 1
+      e[2][k] = prmt(a.y, b2.y, 0x5410u);
+      e[3][k] = prmt(a.y, b2.y, 0x7632u);
     }
-    even[c] = make_uint4(e[0], e[1], e[2], e[3]);
-    odd[c] = make_uint4(o[0], o[1], o[2], o[3]);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) col[j][c] = make_uint4(e[j][0], e[j][1], e[j][2], e[j][3]);
   }
   const int64_t units_per_col = rows / kUnitElems;
 #pragma unroll
-  for (int half = 0; half < 2; ++half) {
+  for (int j = 0; j < 4; ++j) {
     uint32_t codes[4], meta;
-    encode_unit_bf16_pair<kRHA>(half ? odd : even, l, codes, meta);
-    const int64_t col = c0 + 2 * cp + half;
-    if (col < cols) {
-      uint32_t* out = dst + (col * units_per_col + blockIdx.x) * kUnitWords;
+    encode_unit_bf16_pair<kRHA, 16>(col[j], l, codes, meta);
+    const int64_t c = c0 + 4 * cq + j;
+    if (c < cols) {
+      uint32_t* out = dst + (c * units_per_col + blockIdx.x) * kUnitWords;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) st_stream(out + 1 + 2 * c + l, codes[c]);
+      for (int g = 0; g < 4; ++g) st_stream(out + 1 + 2 * g + l, codes[g]);
       if (l == 0) st_stream(out, meta);
     }
   }
@@ -319,8 +332,8 @@ extern "C" hif4_status hif4_quantize_transposed(const void* src, hif4_dtype dt, 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const uint16_t* x = static_cast<const uint16_t*>(src);
   uint32_t* dst = static_cast<uint32_t*>(dst_units);
-  if (mode == HIF4_RHA) quantize_bf16_transposed_kernel<true><<<grid, 128, 0, st>>>(x, rows, cols, ld_src, dst);
-  else quantize_bf16_transposed_kernel<false><<<grid, 128, 0, st>>>(x, rows, cols, ld_src, dst);
+  if (mode == HIF4_RHA) quantize_bf16_transposed_kernel<true><<<grid, kTileThreads, 0, st>>>(x, rows, cols, ld_src, dst);
+  else quantize_bf16_transposed_kernel<false><<<grid, kTileThreads, 0, st>>>(x, rows, cols, ld_src, dst);
   note_launch();
   return launch_status();
 }

@@ -72,10 +72,10 @@ __device__ __forceinline__ uint32_t encode_group_bf16(uint32_t x0, uint32_t x1, 
   return prmt(g0 * 0x1001u, g1 * 0x1001u, 0x7531u);
 }
 
-// One unit held by two consecutive lanes: lane l (0 or 1) holds the level-2 groups l, l + 2, l + 4, l + 6 (16
-// bytes each) in v[0..3].  Returns the lane's four code words (groups l + 2c) and, in both lanes, the
-// unit's metadata word.  Must be called by both lanes of the pair (it exchanges with lane ^ 1).
-template <bool kRHA>
+// One unit held by two lanes, kPartner apart (consecutive by default): lane l (0 or 1) holds the level-2 groups l,
+// l + 2, l + 4, l + 6 (16 bytes each) in v[0..3].  Returns the lane's four code words (groups l + 2c) and, in both
+// lanes, the unit's metadata word.  Must be called by both lanes of the pair (it exchanges with lane ^ kPartner).
+template <bool kRHA, int kPartner = 1>
 __device__ __forceinline__ void encode_unit_bf16_pair(const uint4 (&v)[4], int l, uint32_t (&codes)[4], uint32_t& meta_out) {
   // metadata bit weights of this lane's groups g = 2i + l: E1_8 bit 8 + g, E1_16 bits 16 + 2g, 17 + 2g
   const uint32_t w8 = 0x100u << l, w16 = 0x10000u << (2 * l);
@@ -87,7 +87,7 @@ __device__ __forceinline__ void encode_unit_bf16_pair(const uint4 (&v)[4], int l
   for (int c = 0; c < 4; ++c)
     vm = umax2(vm, umax2(umax2(v[c].x & kAbs, v[c].y & kAbs), umax2(v[c].z & kAbs, v[c].w & kAbs)));
   vm = hmax_halves(vm);
-  vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 1));
+  vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, kPartner));
   const bool unit_nan = vm > 0x7F80u;
 
   // Stage 2: level-1 scale, its reciprocal.
@@ -106,7 +106,7 @@ __device__ __forceinline__ void encode_unit_bf16_pair(const uint4 (&v)[4], int l
     m16 += (e16a + 2u * e16b) << (4 * c);
   }
   uint32_t meta = m8 * w8 + m16 * w16;
-  meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 1);
+  meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, kPartner);
   meta |= byte;
   if (unit_nan) {                                      // NaN unit: E6M2 = NaN, all else zero
     meta = 0xFFu;
