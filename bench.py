@@ -539,6 +539,12 @@ def run_case(spec: str):
         q = torch.empty(n // 4096, 64, 36, dtype=torch.uint8, device=dev)
         fn = lambda: hif4.hif4_quantize_transposed(x, out=q)
         work = f"{n * 2.5625 / 1e6:.1f} MB"
+    elif kind == "quantizeT32":                     # the same from an FP32 source
+        n = 2 ** nums[0]
+        x = wl.quantize_sweep(n, device=dev, dtype=torch.float32).view(4096, n // 4096)
+        q = torch.empty(n // 4096, 64, 36, dtype=torch.uint8, device=dev)
+        fn = lambda: hif4.hif4_quantize_transposed(x, out=q)
+        work = f"{n * 4.5625 / 1e6:.1f} MB"
     elif kind == "quantize16":                      # FP16 source (widened to FP32 inside the kernel)
         n = 2 ** nums[0]
         x = wl.quantize_sweep(n, device=dev).to(torch.float16)
@@ -594,7 +600,7 @@ def main():
     ap.add_argument("--gemm-path", type=int, default=0, help="with --case: kernel selection, see hif4_set_gemm_path")
     ap.add_argument("--case", default=None,
                     help="run one kernel a few times instead of the benchmark (for ncu captures): "
-                         "gemm:M,N,K | quantize:LOG2_ELEMS | dequantize:LOG2_ELEMS | quantize32 / dequantize32 (FP32 side) | quantize16 (FP16 source) | quantizeT (column-wise units) | "
+                         "gemm:M,N,K | quantize:LOG2_ELEMS | dequantize:LOG2_ELEMS | quantize32 / dequantize32 (FP32 side) | quantize16 (FP16 source) | quantizeT / quantizeT32 (column-wise units, BF16 / FP32 source) | "
                          "grouped:TOKENS,EXPERTS,N,K")
     args = ap.parse_args()
     if args.case:

@@ -93,11 +93,11 @@ hif4_status hif4_quantize(const void* src, hif4_dtype dt, int64_t rows, int64_t 
  * vector lies in memory; Eq. 3 needs both GEMM operands cut along the contraction dimension, so a matrix
  * that is contracted along its rows -- a weight kept as [K, N], or any operand of a transposed product --
  * is quantized this way.)
- *   src        device, [rows, cols] BF16, row stride `ld_src` elements (>= cols), rows 16-byte aligned;
- *              rows must be a multiple of 64, cols a multiple of 8.
+ *   src        device, [rows, cols] of `dt` (any source type of hif4_quantize, same working precision), row
+ *              stride `ld_src` elements (>= cols), rows 16-byte aligned; rows must be a multiple of 64, cols
+ *              a multiple of 8.
  *   dst_units  device, cols*(rows/64) units, column-major in the sense above ([cols, rows/64, 36 bytes]),
- *              4-byte aligned.  Fully overwritten.
- * Only HIF4_BF16 sources are built (others return HIF4_ERR_UNSUPPORTED).  */
+ *              4-byte aligned.  Fully overwritten.  */
 hif4_status hif4_quantize_transposed(const void* src, hif4_dtype dt, int64_t rows, int64_t cols,
                                      int64_t ld_src, void* dst_units, hif4_round mode, void* stream);
 

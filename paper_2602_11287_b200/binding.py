@@ -135,7 +135,7 @@ def hif4_quantize(src: torch.Tensor, mode: int = HIF4_RNE, out: Optional[torch.T
 
 def hif4_quantize_transposed(src: torch.Tensor, mode: int = HIF4_RNE, out: Optional[torch.Tensor] = None,
                              stream=None) -> torch.Tensor:
-    """[rows, cols] BF16 -> uint8 units [cols, rows // 64, 36]: the units of src.T without transposing."""
+    """[rows, cols] BF16 / FP32 / FP16 -> uint8 units [cols, rows // 64, 36]: the units of src.T without transposing."""
     _need_cuda(src, out)
     assert src.dim() == 2 and src.stride(1) == 1
     rows, cols = src.shape

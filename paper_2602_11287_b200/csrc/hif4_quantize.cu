@@ -201,6 +201,71 @@ quantize_fp32_kernel(const Src* __restrict__ src, int64_t n_units, int64_t upr, 
   }
 }
 
+// ----------------------------------------------------------------------------- FP32 / FP16 quantizer, units down the columns
+// Same plan as the BF16 kernel above on a tile of 64 rows x 64 columns held as FP32 words (FP16 elements are widened
+// when they are staged): four lanes per unit, lanes l, l + 8, l + 16, l + 24 of a warp, each quad taking four
+// neighbouring columns with one 16-byte load per row (the eight lanes of a quarter warp read 128 consecutive bytes).
+constexpr int kTileCols32 = 64;
+
+template <bool kRHA, typename Src>
+__global__ void __launch_bounds__(kTileThreads)
+quantize_fp32_transposed_kernel(const Src* __restrict__ src, int64_t rows, int64_t cols, int64_t ld_src,
+                                uint32_t* __restrict__ dst) {
+  __shared__ __align__(16) uint32_t tile[kUnitElems * kTileCols32];
+  const int64_t c0 = static_cast<int64_t>(blockIdx.y) * kTileCols32;
+  const int64_t r0 = static_cast<int64_t>(blockIdx.x) * kUnitElems;
+  // 64 rows x 16 chunks of 4 elements; a chunk is inside the matrix or outside as a whole (cols % 8 == 0)
+  constexpr int kChunks = kUnitElems * (kTileCols32 / 4) / kTileThreads;    // 16 per thread
+  uint4 in[kChunks];
+#pragma unroll
+  for (int n = 0; n < kChunks; ++n) {
+    const int i = n * kTileThreads + threadIdx.x, r = i >> 4, ch = i & 15;
+    in[n] = make_uint4(0u, 0u, 0u, 0u);
+    if (c0 + 4 * ch < cols) in[n] = load_group_fp32(src + (r0 + r) * ld_src + c0 + 4 * ch);
+  }
+#pragma unroll
+  for (int n = 0; n < kChunks; ++n) {
+    const int i = n * kTileThreads + threadIdx.x;
+    *reinterpret_cast<uint4*>(tile + 4 * i) = in[n];                         // row i / 16, words 4 (i % 16) ..
+  }
+  __syncthreads();
+  const int lane = threadIdx.x & 31, l = lane >> 3;
+  const int cq = (threadIdx.x >> 5) * 8 + (lane & 7);                        // columns 4 cq .. 4 cq + 3 of the tile
+  uint32_t col[4][4][4];                                                     // [column][group l + 4c][row of the group]
+#pragma unroll
+  for (int c = 0; c < 4; ++c)
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint4 a = *reinterpret_cast<const uint4*>(tile + (4 * (l + 4 * c) + k) * kTileCols32 + 4 * cq);
+      col[0][c][k] = a.x; col[1][c][k] = a.y; col[2][c][k] = a.z; col[3][c][k] = a.w;
+    }
+  const int64_t units_per_col = rows / kUnitElems;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    uint4 v[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) v[c] = make_uint4(col[j][c][0], col[j][c][1], col[j][c][2], col[j][c][3]);
+    uint32_t codes[4], meta;
+    encode_unit_fp32_quad<kRHA, 8>(v, l, codes, meta);
+    const int64_t c = c0 + 4 * cq + j;
+    if (c < cols) {
+      uint32_t* out = dst + (c * units_per_col + blockIdx.x) * kUnitWords;
+      if ((l & 1) == 0) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) st_stream(out + 1 + (l >> 1) + 2 * g, codes[g]);
+      }
+      if (l == 0) st_stream(out, meta);
+    }
+  }
+}
+
+template <typename Src>
+void launch_quantize_fp32_transposed(const Src* x, bool rha, dim3 grid, cudaStream_t st, int64_t rows, int64_t cols,
+                                     int64_t ld_src, uint32_t* dst) {
+  if (rha) quantize_fp32_transposed_kernel<true, Src><<<grid, kTileThreads, 0, st>>>(x, rows, cols, ld_src, dst);
+  else quantize_fp32_transposed_kernel<false, Src><<<grid, kTileThreads, 0, st>>>(x, rows, cols, ld_src, dst);
+}
+
 // ----------------------------------------------------------------------------- dequantizer (Eq. 2)
 // BF16 output: 8 lanes per unit, lane j decodes code word j (elements 8j..8j+7, 16 bytes of output).  FP32 output:
 // 16 lanes per unit, lane k decodes half k & 1 of code word k >> 1 (4 elements, again 16 bytes of output), so that
@@ -324,16 +389,23 @@ extern "C" hif4_status hif4_quantize_transposed(const void* src, hif4_dtype dt, 
   if (rows < 0 || cols < 0 || rows % kUnitElems != 0 || cols % 8 != 0 || ld_src < cols) return HIF4_ERR_SHAPE;
   if (rows == 0 || cols == 0) return HIF4_OK;
   if (!src || !dst_units) return HIF4_ERR_NULL;
-  if (dt != HIF4_BF16) return HIF4_ERR_UNSUPPORTED;
-  if (!aligned(src, 16) || (static_cast<size_t>(ld_src) * 2) % 16 != 0 || !aligned(dst_units, 4)) return HIF4_ERR_ALIGN;
-  const int64_t col_tiles = ceil_div64(cols, kTileCols), row_tiles = rows / kUnitElems;
+  const size_t esz = dt == HIF4_FP32 ? 4 : 2;
+  if (!aligned(src, 16) || (static_cast<size_t>(ld_src) * esz) % 16 != 0 || !aligned(dst_units, 4)) return HIF4_ERR_ALIGN;
+  const int64_t col_tiles = ceil_div64(cols, dt == HIF4_BF16 ? kTileCols : kTileCols32), row_tiles = rows / kUnitElems;
   if (row_tiles > 0x7FFFFFFFll || col_tiles > 65535) return HIF4_ERR_SHAPE;
   const dim3 grid(static_cast<unsigned>(row_tiles), static_cast<unsigned>(col_tiles));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const uint16_t* x = static_cast<const uint16_t*>(src);
   uint32_t* dst = static_cast<uint32_t*>(dst_units);
-  if (mode == HIF4_RHA) quantize_bf16_transposed_kernel<true><<<grid, kTileThreads, 0, st>>>(x, rows, cols, ld_src, dst);
-  else quantize_bf16_transposed_kernel<false><<<grid, kTileThreads, 0, st>>>(x, rows, cols, ld_src, dst);
+  const bool rha = mode == HIF4_RHA;
+  if (dt == HIF4_BF16) {
+    const uint16_t* x = static_cast<const uint16_t*>(src);
+    if (rha) quantize_bf16_transposed_kernel<true><<<grid, kTileThreads, 0, st>>>(x, rows, cols, ld_src, dst);
+    else quantize_bf16_transposed_kernel<false><<<grid, kTileThreads, 0, st>>>(x, rows, cols, ld_src, dst);
+  } else if (dt == HIF4_FP32) {
+    launch_quantize_fp32_transposed(static_cast<const float*>(src), rha, grid, st, rows, cols, ld_src, dst);
+  } else {
+    launch_quantize_fp32_transposed(static_cast<const __half*>(src), rha, grid, st, rows, cols, ld_src, dst);
+  }
   note_launch();
   return launch_status();
 }

@@ -161,10 +161,11 @@ __device__ __forceinline__ uint32_t encode_group_fp32(const uint32_t (&xb)[4], c
   return half;
 }
 
-// One unit held by four consecutive lanes in FP32 bit patterns: lane l (0..3) holds the level-3 groups l, l + 4,
-// l + 8, l + 12 (4 elements each) in v[0..3].  Returns, in the even lanes, the code words (l >> 1) + 2c and, in
-// all four lanes, the unit's metadata word.  Must be called by all four lanes (it exchanges with lane ^ 1, ^ 2).
-template <bool kRHA>
+// One unit held by four lanes, kStride apart (consecutive by default), in FP32 bit patterns: lane l (0..3) holds the
+// level-3 groups l, l + 4, l + 8, l + 12 (4 elements each) in v[0..3].  Returns, in the even lanes, the code words
+// (l >> 1) + 2c and, in all four lanes, the unit's metadata word.  Must be called by all four lanes (it exchanges
+// with lane ^ kStride, ^ 2 kStride).
+template <bool kRHA, int kStride = 1>
 __device__ __forceinline__ void encode_unit_fp32_quad(const uint4 (&v)[4], int l, uint32_t (&codes)[4], uint32_t& meta_out) {
   uint32_t xb[4][4], ab[4][4];
   uint32_t vm = 0u;
@@ -174,8 +175,8 @@ __device__ __forceinline__ void encode_unit_fp32_quad(const uint4 (&v)[4], int l
 #pragma unroll
     for (int e = 0; e < 4; ++e) { ab[c][e] = xb[c][e] & 0x7FFFFFFFu; vm = max(vm, ab[c][e]); }
   }
-  vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 1));
-  vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 2));
+  vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, kStride));
+  vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, 2 * kStride));
   const bool unit_nan = vm > 0x7F800000u;
 
   const float sf = __fmul_rn(__uint_as_float(vm), __uint_as_float(0x3E124925u));   // (1/7)_FP32
@@ -194,7 +195,7 @@ __device__ __forceinline__ void encode_unit_fp32_quad(const uint4 (&v)[4], int l
     const uint32_t p16 = max(max(__float_as_uint(t[0]), __float_as_uint(t[1])),
                              max(__float_as_uint(t[2]), __float_as_uint(t[3])));
     // level-2 peak: this lane's level-3 group and its neighbour's
-    const uint32_t e8 = max(p16, __shfl_xor_sync(0xFFFFFFFFu, p16, 1)) >= 0x40800000u;    // >= 4.0
+    const uint32_t e8 = max(p16, __shfl_xor_sync(0xFFFFFFFFu, p16, kStride)) >= 0x40800000u;    // >= 4.0
     uint32_t e16;
     half[c] = encode_group_fp32<kRHA>(xb[c], t, p16, e8, e16);
     // level-3 group l + 4c -> E1_16 bit 16 + l + 4c; its level-2 group (l >> 1) + 2c -> E1_8 bit, set by the even lane
@@ -203,11 +204,11 @@ __device__ __forceinline__ void encode_unit_fp32_quad(const uint4 (&v)[4], int l
   }
   // even lane: word (l >> 1) + 2c = its four nibbles | the odd neighbour's << 16
   const uint32_t mine01 = half[0] | (half[1] << 16), mine23 = half[2] | (half[3] << 16);
-  const uint32_t other01 = __shfl_xor_sync(0xFFFFFFFFu, mine01, 1), other23 = __shfl_xor_sync(0xFFFFFFFFu, mine23, 1);
+  const uint32_t other01 = __shfl_xor_sync(0xFFFFFFFFu, mine01, kStride), other23 = __shfl_xor_sync(0xFFFFFFFFu, mine23, kStride);
   const uint32_t packed[4] = {(mine01 & 0xFFFFu) | (other01 << 16), (mine01 >> 16) | (other01 & 0xFFFF0000u),
                        (mine23 & 0xFFFFu) | (other23 << 16), (mine23 >> 16) | (other23 & 0xFFFF0000u)};
-  meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 1);
-  meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 2);
+  meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, kStride);
+  meta |= __shfl_xor_sync(0xFFFFFFFFu, meta, 2 * kStride);
   meta |= byte;
 #pragma unroll
   for (int c = 0; c < 4; ++c) codes[c] = unit_nan ? 0u : packed[c];

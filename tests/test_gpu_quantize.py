@@ -240,7 +240,38 @@ def test_quantize_transposed_is_quantize_of_the_transpose(hif4, mode):
         hif4.hif4_quantize_transposed(torch.zeros(100, 64, dtype=torch.bfloat16, device="cuda"))
     assert ei.value.code == 2                                                                      # rows % 64
     with pytest.raises(hif4.Hif4Error) as ei:
-        hif4.hif4_quantize_transposed(torch.zeros(64, 64, dtype=torch.float32, device="cuda"))
-    assert ei.value.code == 8                                                                      # BF16 only
+        hif4.hif4_quantize_transposed(torch.zeros(64, 60, dtype=torch.float32, device="cuda"))
+    assert ei.value.code == 2                                                                      # cols % 8
     assert hif4.hif4_quantize_transposed(torch.zeros(0, 64, dtype=torch.bfloat16, device="cuda")).shape == (64, 0, 36)
+    assert hif4.hif4_last_device_status() == 0
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16])
+def test_quantize_transposed_fp32_and_fp16_sources(hif4, mode, dtype):
+    """Units down the columns of FP32 and FP16 matrices: bit-identical to the oracle's P = FP32 steps on the
+    transposed matrix (ragged column counts, a strided source, special values, values between BF16 neighbours)."""
+    rng = np.random.default_rng(900 + mode)
+    np_dt = np.float32 if dtype == torch.float32 else np.float16
+    cases = []
+    for (rows, cols) in ((64, 8), (128, 72), (640, 1000), (512, 2048)):
+        scale = np.exp2(rng.integers(-12, 12, size=(1, cols))) if dtype == torch.float32 else np.exp2(rng.integers(-6, 6, size=(1, cols)))
+        x = rng.standard_normal((rows, cols)) * scale * np.exp2(-rng.integers(0, 6, size=(rows, cols)))
+        cases.append(x.astype(np_dt))
+    special = rng.standard_normal((256, 256)).astype(np_dt)
+    special[5, 7] = np.nan; special[70, 9] = np.inf; special[130, 11] = -np.inf; special[:, 13] = 0.0
+    special[64:128, 15] = -0.0; special[3, 17] = np.finfo(np_dt).max; special[200, 19] = np.finfo(np_dt).tiny / 4
+    cases.append(special)
+    for x_np in cases:
+        rows, cols = x_np.shape
+        x = torch.from_numpy(x_np).cuda()
+        out = torch.full((cols + 2, rows // 64, 36), 0xCD, dtype=torch.uint8, device="cuda")
+        hif4.hif4_quantize_transposed(x, mode, out=out[1:cols + 1])
+        want = oracle.quantize(np.ascontiguousarray(x_np.T), mode, nthreads=8)
+        _compare_units(out[1:cols + 1].cpu().numpy(), want, f"transposed {dtype} {rows}x{cols} mode {mode}")
+        assert (out[0] == 0xCD).all() and (out[cols + 1] == 0xCD).all()
+        assert torch.equal(out[1:cols + 1], hif4.hif4_quantize(x.t().contiguous(), mode)), "differs from quantizing the transpose"
+    wide = torch.from_numpy(cases[2]).cuda()
+    got = hif4.hif4_quantize_transposed(wide[:, 8:808], mode).cpu().numpy()
+    _compare_units(got, oracle.quantize(np.ascontiguousarray(cases[2][:, 8:808].T), mode, nthreads=8), "transposed, strided")
     assert hif4.hif4_last_device_status() == 0
