@@ -65,6 +65,29 @@ def test_host_only_entry_points(cdll):
     assert cdll.hif4_grouped_gemm_workspace(-1, 10, 64, 64, ctypes.byref(n)) == 2
 
 
+def test_gemm_workspace_follows_the_kernel_choice_and_tile_schedule(cdll):
+    """hif4_gemm_workspace is host logic: it picks the kernel by M and plans the tile schedule.  Sizes worked out
+    by hand for 148 SMs = 74 CTA pairs (what the library assumes without a device, and what a B200 has)."""
+    i64, sz = ctypes.c_int64, ctypes.c_size_t
+    cdll.hif4_gemm_workspace.argtypes = [i64, i64, i64, ctypes.POINTER(sz)]
+    n = sz(0)
+    want = {
+        # M <= 32: decoded activation rows, 2 bytes x K x (8, 16 or 32 rows)
+        (1, 4096, 4096): 2 * 4096 * 8, (16, 14336, 4096): 2 * 4096 * 16, (32, 4096, 14336): 2 * 14336 * 32,
+        # 33..128 rows: 56 weight tiles on 74 pairs are not sliced; 16 tiles x 4 K slices x 8 completion words
+        (64, 14336, 4096): 0, (128, 4096, 14336): 16 * 4 * 8 * 4,
+        # pair kernel, several rounds with a partial one: (74 + 1) flag rows x 2 x 8 words, rounded up to 256 bytes
+        (4096, 14336, 4096): 4864, (4096, 4096, 4096): 4864,
+        # a whole number of rounds, or one round that is not worth slicing: nothing
+        (256 * 74, 256, 1024): 0, (4096, 1024, 4096): 0, (4096, 4096, 192): 0,
+        # one round of 32 tiles x 2 slices, of 8 tiles x 4 slices
+        (2048, 1024, 8192): 32 * 2 * 8 * 4, (1024, 512, 16384): 8 * 4 * 8 * 4,
+    }
+    for (M, N, K), bytes_ in want.items():
+        assert cdll.hif4_gemm_workspace(M, N, K, ctypes.byref(n)) == 0
+        assert n.value == bytes_, (M, N, K, n.value, bytes_)
+
+
 def test_argument_errors_are_found_before_any_launch(cdll):
     """Shape / dtype / null checks come before the first CUDA call, so they answer without a GPU."""
     i64, vp, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
