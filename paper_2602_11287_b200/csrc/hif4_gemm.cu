@@ -32,7 +32,7 @@ extern "C" hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size
     if (few_bytes > *bytes) *bytes = few_bytes;
   }
   if (g_gemm_path == 3 || (g_gemm_path == 0 && M >= kPairMinM)) {
-    const size_t pair_bytes = gemm_tc2_workspace_bytes(M, N, K);     // completion words of a K-sliced last round
+    const size_t pair_bytes = gemm_tc2_workspace_bytes(M, N, K);     // completion words of tiles shared along K
     if (pair_bytes > *bytes) *bytes = pair_bytes;
   }
   return HIF4_OK;

@@ -17,7 +17,7 @@ hif4_status launch_gemm_tc(const void* A, const void* B, float* C, int64_t M, in
                            cudaStream_t st);
 // Tensor-core path on CTA pairs (256 x 256 tiles, tcgen05 cta_group::2): same requirements.
 bool gemm_tc2_supported(const void* A, const void* B, int64_t M, int64_t N, int64_t K);
-// Workspace: completion words of the K-sliced last round of the tile schedule (0 when that round is not split).
+// Workspace: completion words of the tiles that two or more pairs share along K (0 when the schedule splits none).
 size_t gemm_tc2_workspace_bytes(int64_t M, int64_t N, int64_t K);
 hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,
                             void* workspace, size_t workspace_bytes, cudaStream_t st);
