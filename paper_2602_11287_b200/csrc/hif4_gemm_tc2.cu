@@ -78,7 +78,7 @@ struct Gemm2Params {
   // pair, the K = 256 chunks of the remaining `sk_tiles` tiles (between one and two per pair, starting at tile
   // `sk_tile0`), laid end to end, are dealt out in equal contiguous runs.  A run begins with the last chunks of a
   // tile whose first chunks end the previous pair's run: the pair that has the end of a tile computes it first and
-  // stores it (slice 0, flag row = its own index), the pair that has the beginning computes it last and adds
+  // stores it (slice 0, flag row = the index of its run), the pair that has the beginning computes it last and adds
   // (slice 1), so the addition hardly ever waits.
   int sk_tiles;
   int sk_tile0;
@@ -94,11 +94,16 @@ struct WorkItem {
   int tail;             // index among the tail tiles, -1 for a whole tile
   int slice;            // K slice of a tail tile
 };
-// First and last chunk (exclusive) of a pair's run in the balanced rounds, in chunks of the sk_tiles tiles laid end to end.
-__device__ __forceinline__ void balanced_run(const Gemm2Params& p, int pair, int num_pairs, int64_t& c0, int64_t& c1) {
+// First and last chunk (exclusive) of a pair's run in the balanced rounds, in chunks of the sk_tiles tiles laid end to
+// end.  The runs go to the pairs in descending order (`run` = num_pairs - 1 - pair), so that the pair that waits
+// for its neighbour's part of a shared tile has the higher index: CTAs are handed out in index order, and a
+// grid that is only partly resident still cannot wait for a CTA that has not started.
+__device__ __forceinline__ int balanced_run(const Gemm2Params& p, int pair, int num_pairs, int64_t& c0, int64_t& c1) {
   const int64_t total = static_cast<int64_t>(p.sk_tiles) * p.num_kc;
-  c0 = total * pair / num_pairs;
-  c1 = total * (pair + 1) / num_pairs;
+  const int run = num_pairs - 1 - pair;
+  c0 = total * run / num_pairs;
+  c1 = total * (run + 1) / num_pairs;
+  return run;
 }
 __device__ __forceinline__ int num_work_items(const Gemm2Params& p, int pair, int num_pairs) {
   if (p.sk_tiles > 0) {
@@ -116,14 +121,14 @@ __device__ __forceinline__ WorkItem work_item(const Gemm2Params& p, int pair, in
     w.kc0 = 0; w.kc1 = p.num_kc; w.tail = -1; w.slice = 0;
   } else if (p.sk_tiles > 0) {
     int64_t c0, c1;
-    balanced_run(p, pair, num_pairs, c0, c1);
+    const int run = balanced_run(p, pair, num_pairs, c0, c1);
     const int64_t tr = c0 / p.num_kc + (i - p.full_rounds);
     const int64_t first = tr * p.num_kc;
     w.kc0 = c0 > first ? static_cast<int>(c0 - first) : 0;
     w.kc1 = c1 < first + p.num_kc ? static_cast<int>(c1 - first) : p.num_kc;
     t = p.sk_tile0 + static_cast<int>(tr);
-    if (w.kc0 > 0) { w.tail = pair; w.slice = 0; }                       // end of a tile: computed first, stored
-    else if (w.kc1 < p.num_kc) { w.tail = pair + 1; w.slice = 1; }       // beginning of a tile: computed last, added
+    if (w.kc0 > 0) { w.tail = run; w.slice = 0; }                        // end of a tile: computed first, stored
+    else if (w.kc1 < p.num_kc) { w.tail = run + 1; w.slice = 1; }        // beginning of a tile: computed last, added
     else { w.tail = -1; w.slice = 0; }
   } else {
     w.tail = pair % p.tail_tiles;
