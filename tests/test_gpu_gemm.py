@@ -285,6 +285,28 @@ def test_cta_pair_kernel_k_sliced_last_round(hif4, M, N, K):
     assert hif4.hif4_last_device_status() == 0
 
 
+def test_cta_pair_kernel_random_shapes_against_the_single_cta_kernel(hif4):
+    """Seeded random shapes around the schedule's case distinctions (fewer tiles than CTA pairs with and without K
+    slices, whole rounds, a partial round balanced chunk by chunk, ragged edges, K of one to sixteen chunks): every
+    entry against the single-CTA kernel, which never splits a tile, plus sampled entries against FP64."""
+    rng = np.random.default_rng(20260211)
+    shapes = [(int(rng.integers(129, 5000)), int(rng.integers(8, 5000)), 256 * int(rng.integers(1, 17))) for _ in range(14)]
+    shapes += [(256 * 74, 256, 512), (256 * 37, 512, 768), (257, 256 * 74 + 8, 256)]      # exactly one and two rounds, one more tile
+    for M, N, K in shapes:
+        g = torch.Generator(device="cuda"); g.manual_seed(M * 7 + N * 3 + K)
+        a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
+        b = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
+        C = check_sampled(hif4, a, b, f"random shape {M}x{N}x{K}", n=300, seed=M + N)
+        hif4.hif4_set_gemm_path(2)
+        try:
+            C1 = hif4.hif4_gemm(a, b)
+        finally:
+            hif4.hif4_set_gemm_path(0)
+        scale = (C1.abs().max() + 1e-30).item()
+        assert (C - C1).abs().max().item() <= 1e-5 * scale * K, (M, N, K)
+    assert hif4.hif4_last_device_status() == 0
+
+
 def test_tensor_core_kernel_c_rows_not_16_byte_aligned(tc_path):
     """ldc odd and a base that is only 4-byte aligned: the kernels fall back from vector / TMA stores."""
     hif4 = tc_path
