@@ -15,9 +15,13 @@
 // Parity pins (tests/test_oracle_*.py): Table I / Table II constants, exhaustive decode of all
 // 255 x 2 x 2 x 16 combinations against integer arithmetic, hand-derived worked encodings, E6M2
 // rounding vectors, sign/scale/permutation invariants, the paper's Gaussian MSE ratio, brute-force
-// optimum as a lower bound, Eq. 3 against the flat sum.
-// Parity unpinned: the byte/bit order inside a unit and the FP32-source constants are conventions
-// of this repository (the paper's unit figure is not available as text); the paper prints no
+// optimum as a lower bound, Eq. 3 against the flat sum.  The P = FP32 form of Algorithm 1 (FP32 and
+// FP16 sources) is pinned separately: a restatement with numpy float32 products on thousands of
+// units in both rounding modes, and hand-derived cases in which a BF16-precision (1/7), scale
+// product, table entry or threshold product would change a byte, a micro-exponent or a code.
+// Parity unpinned: the byte/bit order inside a unit and the choice of FP32 working precision for
+// FP32/FP16 sources are conventions of this repository (the paper's unit figure is not available
+// as text and it only says that "a similar procedure" applies to those types); the paper prints no
 // worked encoding, so the worked examples are derived by hand from Algorithm 1.
 
 #include <cmath>

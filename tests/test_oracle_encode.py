@@ -360,6 +360,172 @@ def test_oracle_matches_restatement_on_library_bf16_arithmetic():
     assert np.array_equal(np.stack([codes_of(v) for v in u]), codes)
 
 
+# ------------------------------------------------------------------ restatement with library FP32
+def _algorithm1_with_numpy_fp32(x, mode):
+    """Algorithm 1 in its literal order with ``numpy.float32`` products as the arithmetic (each ``*`` of two
+    float32 arrays is one IEEE multiply rounded to nearest-even; scalings by powers of two are exact).
+    Constants: ``np.float32(1/7)`` and ``np.float32(1/1.M)``.  x: float32 ``[n, 64]`` without NaN."""
+    f32 = np.float32
+    rnd = (lambda v: np.floor(v + 0.5)) if mode == oracle.RHA else np.rint
+    n = x.shape[0]
+    a = np.abs(x)
+    V16 = a.reshape(n, 16, 4).max(axis=2)
+    V8 = V16.reshape(n, 8, 2).max(axis=2)
+    Vmax = V8.max(axis=1)
+    with np.errstate(over="ignore", invalid="ignore", under="ignore"):
+        SF = (Vmax * f32(1.0 / 7.0)).astype(np.float64)          # float32 product, widened exactly
+        frac, e = np.frexp(SF)                                     # SF = frac * 2^e, frac in [0.5, 1)
+        q = rnd((frac * 2 - 1) * 4).astype(np.int64)
+        e = e.astype(np.int64) - 1
+        e += q == 4
+        q[q == 4] = 0
+        byte = ((e + 48) << 2) | q
+        byte = np.where((e > 15) | ((e == 15) & (q == 3)) | np.isinf(SF), 0xFE, byte)
+        byte = np.where((SF <= 0) | (e < -48), 0x00, byte).astype(np.int64)
+        E, M = (byte >> 2) - 48, byte & 3
+        table = np.array([f32(1.0), f32(1.0 / 1.25), f32(1.0 / 1.5), f32(1.0 / 1.75)], dtype=f32)
+        REC = (table[M] * np.exp2(-E.astype(np.float64)).astype(f32)).astype(f32)   # power-of-two factor: exact
+        p8 = (V8 * REC[:, None]).astype(np.float64)
+        e8 = (p8 >= 4).astype(np.int64)
+        p16 = (V16 * REC[:, None]).astype(np.float64)
+        e16 = (p16 * 0.5 ** np.repeat(e8, 2, axis=1) >= 2).astype(np.int64)
+        t = np.abs((x * REC[:, None]).astype(np.float64))
+        quarters = t * 4 * 0.5 ** (np.repeat(e8, 8, axis=1) + np.repeat(e16, 4, axis=1))
+        mag = np.minimum(rnd(quarters), 7).astype(np.uint8)
+    codes = mag | (np.signbit(x).astype(np.uint8) << 3)
+    meta = byte.astype(np.uint32)
+    meta |= (e8 << (8 + np.arange(8))).sum(axis=1).astype(np.uint32)
+    meta |= (e16 << (16 + np.arange(16))).sum(axis=1).astype(np.uint32)
+    return meta, codes
+
+
+def _fp32_pin_inputs():
+    from tests import adversarial
+    rng = np.random.default_rng(16)
+    chunks = [rng.standard_t(4, (700, 64)), rng.standard_normal((700, 64)), rng.uniform(-1, 1, (400, 64))]
+    spike = rng.standard_normal((300, 64))
+    spike[np.arange(300), rng.integers(0, 64, 300)] *= 1000
+    chunks.append(spike)
+    chunks.append(rng.standard_normal((400, 64)) * np.exp2(rng.integers(-70, 40, (400, 1))))
+    # peaks placed next to every E6M2 rounding boundary: Vmax ~ 7 * (1.125, 1.375, 1.625, 1.875) * 2^k
+    edge = rng.standard_normal((800, 64)) * 0.3
+    ties = np.array([1.125, 1.375, 1.625, 1.875])[rng.integers(0, 4, 800)]
+    edge[np.arange(800), rng.integers(0, 64, 800)] = 7 * ties * np.exp2(rng.integers(-3, 3, 800)) * \
+        (1 + rng.integers(-3, 4, 800) * 2.0 ** -23)
+    chunks.append(edge)
+    x = np.concatenate(chunks).astype(np.float32)
+    adv = adversarial.fp32_adversarial(seed=5, n_units=1500)
+    adv = adv[~np.isnan(adv).any(axis=1)]
+    return np.concatenate([x, adv])
+
+
+@pytest.mark.parametrize("mode", [oracle.RNE, oracle.RHA])
+def test_oracle_matches_restatement_on_library_fp32_arithmetic(mode):
+    x = _fp32_pin_inputs()
+    assert x.shape[0] >= 4000
+    u = oracle.quantize(x, mode)[:, 0]
+    meta, codes = _algorithm1_with_numpy_fp32(x, mode)
+    assert np.array_equal(u[:, :4].copy().view("<u4")[:, 0], meta)
+    got = np.empty((u.shape[0], 64), dtype=np.uint8)
+    got[:, 0::2] = u[:, 4:] & 0xF
+    got[:, 1::2] = u[:, 4:] >> 4
+    assert np.array_equal(got, codes)
+
+
+@pytest.mark.parametrize("mode", [oracle.RNE, oracle.RHA])
+def test_fp16_sources_match_the_fp32_restatement_on_widened_values(mode):
+    rng = np.random.default_rng(17)
+    x = (rng.standard_t(4, (1500, 64)) * np.exp2(rng.integers(-20, 12, (1500, 1)))).astype(np.float16)
+    x[0, :] = np.float16(6.0e-8)            # subnormals
+    x[1, 3] = np.float16(65504.0)
+    x[2, 9] = np.float16(-np.inf)
+    u = oracle.quantize(x, mode)[:, 0]
+    meta, codes = _algorithm1_with_numpy_fp32(x.astype(np.float32), mode)
+    assert np.array_equal(u[:, :4].copy().view("<u4")[:, 0], meta)
+    got = np.empty((u.shape[0], 64), dtype=np.uint8)
+    got[:, 0::2] = u[:, 4:] & 0xF
+    got[:, 1::2] = u[:, 4:] >> 4
+    assert np.array_equal(got, codes)
+
+
+# ------------------------------------------------------------------ FP32 hand cases where BF16 constants differ
+def _enc_fp32(pairs, mode=oracle.RNE):
+    x = np.zeros((1, 64), dtype=np.float32)
+    for i, v in pairs.items():
+        x[0, i] = v
+    assert all(float(x[0, i]) == v for i, v in pairs.items()), "hand-case values must be exact in FP32"
+    u = oracle.quantize(x, mode)[0, 0]
+    return meta_of(u), codes_of(u)
+
+
+def test_fp32_hand_case_scale_product_is_rounded_to_fp32_with_the_fp32_seventh():
+    """Peak 7.875 alone.  (1/7)_FP32 = 0x3E124925 = 9586981 * 2^-26, so the exact product is
+    7.875 * 9586981 * 2^-26 = 1.125 + 27 * 2^-29 (63 * 9586981 = 603979803 = 9 * 2^26 + 27, over 2^29).
+    FP32 spacing at 1.125 is 2^-23 = 64 * 2^-29, so the product rounds to exactly 1.125: a tie of the 3-bit
+    significand.  Half-to-even gives 1.0 (byte 0xC0, REC = 1, peak scaled 7.875 / 4 = 1.96875 -> 7.875 quarters ->
+    8 -> clamped to 7); half-away gives 1.25 (byte 0xC1, REC = fl32(0.8), 7.875 * 0.8 = 6.3 -> /4 -> 6.3 quarters ->
+    code 6).  An unrounded product (1.125 + 27 * 2^-29, above the tie) would give 0xC1 in both modes, and the BF16
+    seventh 0.142578125 gives 1.1228 -> 0xC0 in both modes: only a product rounded once to FP32 tells the modes
+    apart here."""
+    m, c = _enc_fp32({40: 7.875}, oracle.RNE)
+    assert m == (0xC0 | (1 << (8 + 5)) | (1 << (16 + 10))) and c[40] == 7
+    m, c = _enc_fp32({40: 7.875}, oracle.RHA)
+    assert m == (0xC1 | (1 << (8 + 5)) | (1 << (16 + 10))) and c[40] == 6
+
+
+def test_fp32_hand_case_scale_is_not_narrowed_to_bf16():
+    """Peak 7.8828125 = 1009 / 128 alone.  Product with (1/7)_FP32: 1009 * 9586981 * 2^-33 = 1.12611607...,
+    above the tie 1.125 -> significand 1.25 -> byte 0xC1 in both modes.  Narrowing that scale to BF16 first
+    (spacing 2^-7 at 1: neighbours 1.125 and 1.1328125) would land on the tie 1.125 and half-to-even would give
+    0xC0.  With 0xC1: REC = fl32(0.8) = 0.800000012; 7.8828125 * REC = 6.30625009 -> both micro-exponents ->
+    6.30625 quarters -> code 6."""
+    for mode in (oracle.RNE, oracle.RHA):
+        m, c = _enc_fp32({0: -7.8828125}, mode)
+        assert m == (0xC1 | (1 << 8) | (1 << 16)) and c[0] == 0x8 | 6
+
+
+def test_fp32_hand_case_level2_threshold_is_compared_in_fp32():
+    """Peak 7 in group 0 (7 * (1/7)_FP32 = 1 + 3 * 2^-26 rounds to 1.0 -> byte 0xC0, REC = 1) and 3.99609375 =
+    1023 / 256 in group 3 (elements 24..31).  In FP32 the product with REC = 1 is 3.99609375 < 4, so E1_8[3] = 0;
+    it is >= 2, so E1_16[6] = 1, and the element scales to 1.998046875 -> 7.99 quarters -> 8 -> clamped to 7.
+    A BF16 product (spacing 2^-6 in [2, 4): neighbours 3.984375 and 4.0, the value lies 3/4 of the way up) would be
+    4.0, set E1_8[3], and the code would become 3.99609375 quarters -> 4."""
+    m, c = _enc_fp32({0: 7.0, 24: 3.99609375})
+    assert m == (0xC0 | (1 << 8) | (1 << 16) | (1 << (16 + 6)))
+    assert c[0] == 7 and c[24] == 7
+
+
+def test_fp32_hand_case_level3_threshold_is_compared_in_fp32():
+    """Peak 7 in group 0 (byte 0xC0, REC = 1, as above) and 1.998046875 = 1023 / 512 at element 24.  FP32 product
+    1.998046875 < 2: neither micro-exponent of that element is set, it stays 7.99 quarters -> 8 -> clamped to 7.
+    A BF16 product (spacing 2^-7 in [1, 2)) would be 2.0, set E1_16[6], and the code would be 3.996 quarters -> 4."""
+    m, c = _enc_fp32({0: 7.0, 24: 1.998046875})
+    assert m == (0xC0 | (1 << 8) | (1 << 16))
+    assert c[0] == 7 and c[24] == 7
+
+
+def test_fp32_hand_cases_reciprocal_table_entries_are_fp32():
+    """M = 1: peak 1.0 -> SF = (1/7)_FP32 = 1.142857 * 2^-3 -> significand 1.25 -> byte 0xB5, REC = fl32(0.8) * 8 =
+    0x3F4CCCCD * 8 = 6.4000001.  Element 1919 / 32768 = 0.058563232421875: times 6.4000001 = 0.3748047 ->
+    1.49922 quarters -> code 1.  The BF16 entry 0x3F4D (0.80078125, REC 6.40625) would give 0.3751707 ->
+    1.50068 quarters -> code 2.
+    M = 2: peak 10.5 -> exact product 21 * 9586981 * 2^-27 = 1.5 + 9 * 2^-27, which FP32 (spacing 16 * 2^-27)
+    rounds to 1.5 + 2^-23: significand 1.5 either way -> byte 0xC2, REC = fl32(2/3) = 0x3F2AAAAB =
+    0.66666669.  Element 0.5615234375 = 575 / 1024: times 0.66666669 = 0.37434897 -> 1.49740 quarters -> code 1.
+    The BF16 entry 0x3F2B (0.66796875) would give 0.375080 -> 1.50032 quarters -> code 2.
+    M = 3: peak 12.25 -> exact product 49 * 9586981 * 2^-28 = 1.75 + 21 * 2^-28 -> FP32 1.75 + 2^-23 -> significand
+    1.75 -> byte 0xC3, REC = fl32(4/7) = 0x3F124925 = 0.5714286.
+    Element 0.65625 = 21 / 32: times 0.5714286 = 0.37500002 -> above the tie 1.5 quarters -> code 2 in both modes.
+    The BF16 entry 0x3F12 (0.5703125) would give 0.37426758 -> 1.49707 quarters -> code 1."""
+    for mode in (oracle.RNE, oracle.RHA):
+        m, c = _enc_fp32({0: 1.0, 8: 0.058563232421875}, mode)
+        assert (m & 0xFF) == 0xB5 and c[0] == 6 and c[8] == 1
+        m, c = _enc_fp32({0: 10.5, 8: 0.5615234375}, mode)
+        assert (m & 0xFF) == 0xC2 and c[0] == 7 and c[8] == 1
+        m, c = _enc_fp32({0: 12.25, 8: 0.65625}, mode)
+        assert (m & 0xFF) == 0xC3 and c[0] == 7 and c[8] == 2
+
+
 # ------------------------------------------------------------------ idempotence on the canonical class
 def test_reencoding_decoded_units_is_stable_where_algorithm1_guarantees_it():
     """decode(encode(decode(u))) == decode(u) for units that Algorithm 1 itself can emit with their
