@@ -27,10 +27,11 @@ UNIT_ELEMS, UNIT_BYTES = 64, 36
 def build(force: bool = False) -> str:
     """Compile the oracle with g++ (no fast-math, no FMA contraction) and return the .so path."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = f"{_LIB}.{os.getpid()}.tmp"       # several processes may build at once: each its own file, then an atomic rename
         cmd = ["g++", "-O2", "-std=c++17", "-fPIC", "-shared", "-ffp-contract=off", "-fno-fast-math",
-               "-pthread", "-Wall", "-Wextra", "-o", _LIB + ".tmp", _SRC]
+               "-pthread", "-Wall", "-Wextra", "-o", tmp, _SRC]
         subprocess.run(cmd, check=True)
-        os.replace(_LIB + ".tmp", _LIB)
+        os.replace(tmp, _LIB)
     return _LIB
 
 
