@@ -597,7 +597,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch the decode-shaped linears directly instead of replaying a CUDA graph")
-    ap.add_argument("--gemm-path", type=int, default=0, help="with --case: kernel selection, see hif4_set_gemm_path")
+    ap.add_argument("--gemm-path", type=int, default=0, help="with --case: kernel selection, see hif4_debug_set_gemm_path")
     ap.add_argument("--case", default=None,
                     help="run one kernel a few times instead of the benchmark (for ncu captures): "
                          "gemm:M,N,K | quantize:LOG2_ELEMS | dequantize:LOG2_ELEMS | quantize32 / dequantize32 (FP32 side) | quantize16 (FP16 source) | quantizeT / quantizeT32 (column-wise units, BF16 / FP32 source) | "
@@ -606,7 +606,7 @@ def main():
     if args.case:
         if args.gemm_path:
             import paper_2602_11287_b200 as hif4
-            hif4.hif4_set_gemm_path(args.gemm_path)
+            hif4.hif4_debug_set_gemm_path(args.gemm_path)
         run_case(args.case)
         return
     if args.impl == "reference":

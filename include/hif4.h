@@ -110,7 +110,8 @@ hif4_status hif4_dequantize(const void* src_units, int64_t rows, int64_t cols, v
 
 /* Workspace (device scratch) that hif4_gemm needs for this shape on the current device; may be 0.
  * For M <= 32 it holds the decoded activation rows (2 * K * 8, 16 or 32 bytes); for larger M a few KB of
- * completion words when tiles are split along K.  Host-only.  */
+ * completion words when tiles are split along K.  The figure is the largest need over all kernels that
+ * could serve the shape, so it stays valid whatever path is chosen at call time.  Host-only.  */
 hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size_t* bytes);
 
 /* hif4_gemm -- C = A * B^T with A, B in HiF4 and FP32 accumulation: C[i][j] is the sum over the
@@ -168,7 +169,9 @@ hif4_status hif4_grouped_gemm(const void* A_units, const void* B_units, float* C
  * the library; every GPU that loads the library holds it until the process exits.  The call itself
  * performs no cudaMalloc / cudaFree and uses no allocating library routine.
  *
- *   Arguments and result are those of hif4_grouped_gemm (same kernels, same bits in C).
+ *   Arguments are those of hif4_grouped_gemm.  The result meets the same tolerance; it comes from the
+ *   single-CTA tensor-core kernel (128-row tiles), whereas hif4_grouped_gemm normally runs the CTA-pair
+ *   kernel, so the FP32 summation order and therefore the last bits of C may differ between the two.
  *   Limit     ceil(total_rows / 128) + num_groups table entries of 16 bytes, rounded up to 256,
  *             must fit in HIF4_NOALLOC_SCRATCH_BYTES (65536: e.g. 256 groups and 491520 rows);
  *             beyond that the call returns HIF4_ERR_WORKSPACE and launches nothing.
@@ -179,7 +182,7 @@ hif4_status hif4_grouped_gemm(const void* A_units, const void* B_units, float* C
  *   Set-up    the first call on each GPU looks up the array's device address
  *             (cudaGetSymbolAddress, with that GPU current) and keeps it; make that first call
  *             outside any stream capture.
- * hif4_set_gemm_path does not apply to this call.  */
+ * hif4_debug_set_gemm_path does not apply to this call.  */
 #define HIF4_NOALLOC_SCRATCH_BYTES 65536
 hif4_status hif4_grouped_gemm_noalloc(const void* A_units, const void* B_units, float* C,
                                       const int64_t* group_offsets_dev, int num_groups,
@@ -197,15 +200,28 @@ hif4_status hif4_last_device_status(void* stream);
 /* Static, NUL-terminated description of a status code.  Host-only.  */
 const char* hif4_status_string(hif4_status s);
 
-/* Diagnostic: 0 = choose the GEMM kernel by shape (default), 1 = CUDA-core kernel only, 2 = the
- * single-CTA tensor-core (tcgen05) kernel whenever it is legal (K % 256 == 0, 16-byte aligned
- * operands), even for small M, 3 = the CTA-pair tensor-core kernel (256 x 256 tiles) whenever it is
- * legal, 4 = the weight-streaming kernel whenever it is legal (M <= 32).  Process-wide, not
- * thread-safe; meant for tests and benchmarks.  */
-hif4_status hif4_set_gemm_path(int path);
+/* ---------------------------------------------------------------------------------------------
+ * Test and benchmark hooks (hif4_debug_*).  Not part of the product surface: nothing above depends on
+ * them except that hif4_gemm honours the path override while it is set.
+ *
+ * hif4_debug_set_gemm_path: 0 = choose the GEMM kernel by shape (default), 1 = CUDA-core kernel only,
+ * 2 = the single-CTA tensor-core (tcgen05) kernel whenever it is legal (K % 256 == 0, 16-byte aligned
+ * operands), even for small M, 3 = the CTA-pair tensor-core kernel (256 x 256 tiles) whenever it is legal,
+ * 4 = the weight-streaming kernel whenever it is legal (M <= 32).  Process-wide and not thread-safe.
+ * hif4_gemm_workspace does not depend on it: it always reports the largest need over all paths.
+ *
+ * hif4_debug_launch_count: number of kernels this library has launched in this process (monotonic,
+ * host-side counter).  */
+hif4_status hif4_debug_set_gemm_path(int path);
+uint64_t hif4_debug_launch_count(void);
 
-/* Number of kernels this library has launched in this process (monotonic, host-side counter).  */
-uint64_t hif4_launch_count(void);
+/* hif4_debug_wait_timeout: launches a one-block kernel that waits on an mbarrier nobody arrives on, with the
+ * same bounded-wait helper the GEMM kernels use but a budget of `budget_ns` (1 .. 100 000 000) instead of their
+ * 2 s.  The wait runs out, the kernel raises the device error word and returns normally; the next
+ * hif4_last_device_status on that stream returns HIF4_ERR_DEVICE_TIMEOUT, the one after it HIF4_OK.  Nothing
+ * faults or hangs: no copy or MMA is in flight.  (The paper has no counterpart; this exercises the library's
+ * failure reporting.)  */
+hif4_status hif4_debug_wait_timeout(uint64_t budget_ns, void* stream);
 
 #ifdef __cplusplus
 }

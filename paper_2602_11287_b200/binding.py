@@ -23,8 +23,8 @@ HIF4_OK = 0
 EXPORTED_SYMBOLS = [
     "hif4_packed_bytes", "hif4_quantize", "hif4_dequantize", "hif4_gemm_workspace", "hif4_gemm",
     "hif4_grouped_gemm_workspace", "hif4_grouped_gemm", "hif4_last_device_status", "hif4_status_string",
-    "hif4_launch_count", "hif4_set_gemm_path", "hif4_grouped_gemm_noalloc", "hif4_grouped_gemm_noalloc_capacity",
-    "hif4_linear", "hif4_linear_workspace", "hif4_quantize_transposed",
+    "hif4_debug_launch_count", "hif4_debug_set_gemm_path", "hif4_grouped_gemm_noalloc", "hif4_grouped_gemm_noalloc_capacity",
+    "hif4_linear", "hif4_linear_workspace", "hif4_quantize_transposed", "hif4_debug_wait_timeout",
 ]
 
 
@@ -69,10 +69,12 @@ def _load() -> ctypes.CDLL:
     L.hif4_last_device_status.argtypes = [vp]
     L.hif4_status_string.restype = ctypes.c_char_p
     L.hif4_status_string.argtypes = [ci]
-    L.hif4_set_gemm_path.restype = ci
-    L.hif4_set_gemm_path.argtypes = [ci]
-    L.hif4_launch_count.restype = ctypes.c_uint64
-    L.hif4_launch_count.argtypes = []
+    L.hif4_debug_set_gemm_path.restype = ci
+    L.hif4_debug_set_gemm_path.argtypes = [ci]
+    L.hif4_debug_launch_count.restype = ctypes.c_uint64
+    L.hif4_debug_launch_count.argtypes = []
+    L.hif4_debug_wait_timeout.restype = ci
+    L.hif4_debug_wait_timeout.argtypes = [ctypes.c_uint64, vp]
     return L
 
 
@@ -111,7 +113,7 @@ def _need_cuda(*tensors: torch.Tensor) -> None:
 
 
 def launch_count() -> int:
-    return int(lib.hif4_launch_count())
+    return int(lib.hif4_debug_launch_count())
 
 
 def hif4_packed_bytes(rows: int, cols: int) -> int:
@@ -282,9 +284,15 @@ def hif4_grouped_gemm_noalloc(a_units: torch.Tensor, b_units: torch.Tensor, grou
     return out
 
 
-def hif4_set_gemm_path(path: int) -> None:
-    """0 = by shape, 1 = CUDA-core kernel only, 2 = tensor-core kernel whenever legal."""
-    _check("hif4_set_gemm_path", lib.hif4_set_gemm_path(path))
+def hif4_debug_set_gemm_path(path: int) -> None:
+    """Test hook: 0 = by shape, 1 = CUDA-core kernel, 2 = single-CTA tensor-core kernel, 3 = CTA-pair kernel,
+    4 = weight-streaming kernel (each whenever legal)."""
+    _check("hif4_debug_set_gemm_path", lib.hif4_debug_set_gemm_path(path))
+
+
+def hif4_debug_wait_timeout(budget_ns: int, stream=None) -> None:
+    """Test hook: a kernel whose bounded wait (budget_ns) runs out on purpose; see include/hif4.h."""
+    _check("hif4_debug_wait_timeout", lib.hif4_debug_wait_timeout(int(budget_ns), _stream(stream)))
 
 
 def hif4_last_device_status(stream=None) -> int:

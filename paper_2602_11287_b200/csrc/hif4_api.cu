@@ -42,7 +42,7 @@ extern "C" const char* hif4_status_string(hif4_status s) {
   return "unknown status";
 }
 
-extern "C" uint64_t hif4_launch_count(void) { return hif4::g_launches.load(std::memory_order_relaxed); }
+extern "C" uint64_t hif4_debug_launch_count(void) { return hif4::g_launches.load(std::memory_order_relaxed); }
 
 extern "C" hif4_status hif4_last_device_status(void* stream) {
   if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return HIF4_ERR_CUDA;

@@ -5,11 +5,12 @@
 using namespace hif4;
 
 namespace {
-// 0 = choose by shape, 1 = CUDA-core kernel only, 2 = single-CTA tensor-core kernel whenever it is
-// legal, 3 = CTA-pair tensor-core kernel whenever it is legal, 4 = weight-streaming kernel whenever
-// it is legal (M <= 16).
+// Test hook (hif4_debug_set_gemm_path): 0 = choose by shape, 1 = CUDA-core kernel only, 2 = single-CTA
+// tensor-core kernel whenever it is legal, 3 = CTA-pair tensor-core kernel whenever it is legal,
+// 4 = weight-streaming kernel whenever it is legal (M <= kGemvMaxM).
 int g_gemm_path = 0;
 constexpr int64_t kPairMinM = 129;      // below that a 256-row pair tile would be half empty
+constexpr int64_t kGroupedMaxRows = (1ll << 31) - 257;   // tile tables keep row numbers (and row + tile height) in 32-bit ints
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -26,19 +27,20 @@ hif4_status check_common(const void* A, const void* B, const float* C, int64_t M
 extern "C" hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size_t* bytes) {
   if (!bytes) return HIF4_ERR_NULL;
   if (M < 0 || N < 0 || K < 0 || K % kUnitElems != 0) return HIF4_ERR_SHAPE;
-  *bytes = gemv_workspace_bytes(M, K);       // decoded tokens of the weight-streaming path (M <= 16)
-  if (g_gemm_path == 0 && M > kGemvMaxM && M < kPairMinM) {
-    const size_t few_bytes = gemm_tc2_swapped_workspace_bytes(M, N, K);  // completion words of the K slices
+  // The largest need over every kernel that may serve this shape, whatever the path override says at call
+  // time: decoded tokens of the weight-streaming path (M <= kGemvMaxM), completion words of the K slices of
+  // the swapped pair kernel (few rows) and of the tiles that the pair kernel shares along K.
+  *bytes = gemv_workspace_bytes(M, K);
+  if (M > kGemvMaxM && M < kPairMinM) {
+    const size_t few_bytes = gemm_tc2_swapped_workspace_bytes(M, N, K);
     if (few_bytes > *bytes) *bytes = few_bytes;
   }
-  if (g_gemm_path == 3 || (g_gemm_path == 0 && M >= kPairMinM)) {
-    const size_t pair_bytes = gemm_tc2_workspace_bytes(M, N, K);     // completion words of tiles shared along K
-    if (pair_bytes > *bytes) *bytes = pair_bytes;
-  }
+  const size_t pair_bytes = gemm_tc2_workspace_bytes(M, N, K);
+  if (pair_bytes > *bytes) *bytes = pair_bytes;
   return HIF4_OK;
 }
 
-extern "C" hif4_status hif4_set_gemm_path(int path) {
+extern "C" hif4_status hif4_debug_set_gemm_path(int path) {
   if (path < 0 || path > 4) return HIF4_ERR_DTYPE;
   g_gemm_path = path;
   return HIF4_OK;
@@ -78,7 +80,8 @@ extern "C" hif4_status hif4_gemm(const void* A_units, const void* B_units, float
 extern "C" hif4_status hif4_grouped_gemm_workspace(int num_groups, int64_t total_rows, int64_t N, int64_t K,
                                                    size_t* bytes) {
   if (!bytes) return HIF4_ERR_NULL;
-  if (num_groups < 0 || total_rows < 0 || N < 0 || K < 0 || K % kUnitElems != 0) return HIF4_ERR_SHAPE;
+  if (num_groups < 0 || total_rows < 0 || total_rows > kGroupedMaxRows || N < 0 || K < 0 || K % kUnitElems != 0)
+    return HIF4_ERR_SHAPE;
   // the tensor-core path keeps its tile table (one 16-byte entry per 128-row tile) here
   *bytes = (K > 0 && K % 256 == 0 && total_rows > 0 && num_groups > 0) ? grouped_tc_workspace_bytes(num_groups, total_rows) : 0;
   return HIF4_OK;
@@ -88,7 +91,7 @@ extern "C" hif4_status hif4_grouped_gemm(const void* A_units, const void* B_unit
                                          const int64_t* group_offsets_dev, int num_groups, int64_t total_rows,
                                          int64_t N, int64_t K, int64_t ldc, void* workspace,
                                          size_t workspace_bytes, void* stream) {
-  if (num_groups < 0) return HIF4_ERR_SHAPE;
+  if (num_groups < 0 || total_rows > kGroupedMaxRows) return HIF4_ERR_SHAPE;
   const hif4_status chk = check_common(A_units, B_units, C, total_rows, N, K, ldc);
   if (chk != HIF4_OK || total_rows == 0 || N == 0 || num_groups == 0) return chk;
   if (!group_offsets_dev) return HIF4_ERR_NULL;

@@ -1,4 +1,4 @@
-// Decode-shaped HiF4 GEMM (M <= 16 tokens): C = A * B^T with the weight matrix B streamed once from
+// Decode-shaped HiF4 GEMM (M <= 32 tokens): C = A * B^T with the weight matrix B streamed once from
 // HBM.  The few tokens are decoded once; the work per weight element is the register decode, so the
 // kernel is organised around decoding with as few instructions per element as possible and around
 // giving every SM the same number of weight rows.
@@ -124,7 +124,7 @@ gemv_prepare_tokens_kernel(const uint32_t* __restrict__ A, int M, int m_pad, int
 
 // The same preparation straight from BF16 activations: Algorithm 1 (the streaming quantizer's own code, two
 // lanes per unit) followed by Eq. 2 of the unit just encoded, without the packed units ever going to memory.
-// Used by the one-call linear layer for M <= 16 BF16 rows; the tokens written are bit-identical to quantizing first.
+// Used by the one-call linear layer for M <= 32 BF16 rows; the tokens written are bit-identical to quantizing first.
 template <bool kRHA>
 __global__ void __launch_bounds__(128)
 gemv_quantize_tokens_kernel(const uint16_t* __restrict__ X, int64_t ld_x, int M, int m_pad, int64_t upr,

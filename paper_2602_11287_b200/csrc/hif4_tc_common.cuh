@@ -49,7 +49,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // Roles that wait long (a whole tile, a whole raw chunk) pass `sleep_ns` > 0 and back off between
 // polls, so that their spinning does not take issue slots from the decode warps.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t sleep_ns = 0) {
+                                          uint32_t sleep_ns = 0, uint64_t budget_ns = kWaitBudgetNs) {
   if (mbar_try(bar, parity)) return true;
   const uint64_t t0 = global_ns();
   for (uint32_t it = 1;; ++it) {
@@ -57,7 +57,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (sleep_ns) __nanosleep(sleep_ns);
     if ((it & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitBudgetNs) {
+      if (global_ns() - t0 > budget_ns) {
         *abort_flag = 1u;
         return false;
       }
@@ -238,14 +238,15 @@ bool make_unit_map(CUtensorMap* map, const void* base, int64_t rows, int64_t upr
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// SM count of the current device (cached per device ordinal: a process may drive several GPUs).
 int sm_count() {
-  static int n = [] {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
-    return v;
-  }();
-  return n;
+  static int cache[64] = {};
+  int dev = 0, v = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (dev >= 0 && dev < 64 && cache[dev] > 0) return cache[dev];
+  if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+  if (dev >= 0 && dev < 64) cache[dev] = v;
+  return v;
 }
 
 }  // namespace

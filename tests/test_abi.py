@@ -92,8 +92,8 @@ def test_argument_errors_are_found_before_any_launch(cdll):
     """Shape / dtype / null checks come before the first CUDA call, so they answer without a GPU."""
     i64, vp, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
     cdll.hif4_quantize.argtypes = [vp, ci, i64, i64, i64, vp, ci, vp]
-    cdll.hif4_launch_count.restype = ctypes.c_uint64
-    before = cdll.hif4_launch_count()
+    cdll.hif4_debug_launch_count.restype = ctypes.c_uint64
+    before = cdll.hif4_debug_launch_count()
     assert cdll.hif4_quantize(None, 0, 4, 100, 100, None, 0, None) == 2     # cols % 64
     assert cdll.hif4_quantize(None, 5, 4, 128, 128, None, 0, None) == 4     # dtype
     assert cdll.hif4_quantize(None, 0, 4, 128, 128, None, 9, None) == 4     # rounding mode
@@ -103,4 +103,4 @@ def test_argument_errors_are_found_before_any_launch(cdll):
     cdll.hif4_gemm.argtypes = [vp, vp, vp, i64, i64, i64, i64, vp, ctypes.c_size_t, vp]
     assert cdll.hif4_gemm(None, None, None, 4, 4, 100, 4, None, 0, None) == 2
     assert cdll.hif4_gemm(None, None, None, 0, 4, 64, 4, None, 0, None) == 0
-    assert cdll.hif4_launch_count() == before
+    assert cdll.hif4_debug_launch_count() == before

@@ -60,6 +60,69 @@ def _sampled_entries(hif4, a_units, b_units, C, what, n=300, seed=0):
     assert np.all(err <= TOL * refabs + 1e-300), f"{what}: worst ratio {np.max(err / np.maximum(TOL * refabs, 1e-300)):.3g}"
 
 
+def _abs_bound_on_device(hif4, a_units, b_units):
+    """sum_k |a_ik| |b_jk| for every entry, formed on the GPU from the decoded operands (FP32 matmul of magnitudes):
+    only the scale of a tolerance between two GPU kernels, never an expected value."""
+    a = hif4.hif4_dequantize(a_units, torch.float32).abs_()
+    b = hif4.hif4_dequantize(b_units, torch.float32).abs_()
+    prev = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = False
+    try:
+        return a @ b.t()
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = prev
+
+
+def _whole_c_against_the_single_cta_kernel(hif4, a_units, b_units, C, what):
+    """Every entry of the default path's C against the single-CTA tensor-core kernel's C (another tile shape, no
+    tile shared between CTAs, another summation order): the two may differ by FP32 rounding only."""
+    hif4.hif4_debug_set_gemm_path(2)
+    try:
+        other = hif4.hif4_gemm(a_units, b_units)
+    finally:
+        hif4.hif4_debug_set_gemm_path(0)
+    bound = _abs_bound_on_device(hif4, a_units, b_units).mul_(2 * TOL)
+    bad = (C - other).abs_() > bound
+    assert not bool(bad.any()), f"{what}: {int(bad.sum())} entries differ between the pair kernel and the single-CTA kernel"
+
+
+def _tile_against_oracle(hif4, a_units, b_units, C, m0, n0, what, rows=256, cols=256):
+    """Every entry of C[m0:m0+rows, n0:n0+cols] against the oracle's FP64 product of those operand rows."""
+    M, N = C.shape
+    m1, n1 = min(M, m0 + rows), min(N, n0 + cols)
+    ref, refabs = oracle.gemm_f64(a_units[m0:m1].cpu().numpy(), b_units[n0:n1].cpu().numpy(), nthreads=oracle.hardware_threads())
+    err = np.abs(C[m0:m1, n0:n1].cpu().numpy().astype(np.float64) - ref)
+    assert np.all(err <= TOL * refabs + 1e-300), f"{what} tile ({m0}, {n0}): worst ratio {np.max(err / np.maximum(TOL * refabs, 1e-300)):.3g}"
+
+
+def _shared_tiles(M, N, pairs=74):
+    """Origins of two 256 x 256 tiles that the balanced last rounds of the pair kernel split between two CTA pairs
+    (the end of the tile stored by one pair, its beginning added by the next), for a device with `pairs` CTA pairs:
+    tiles are numbered row-major; after floor(tiles / pairs) - 1 whole rounds the remaining tiles are dealt out in
+    equal runs of K chunks, so all but a few of them are shared.  Also the last tile of the last row and column."""
+    nt = -(-N // 256)
+    tiles = -(-M // 256) * nt
+    first = (tiles // pairs - 1) * pairs if tiles >= pairs and tiles % pairs else 0
+    picks = [first + 1, (first + tiles) // 2, tiles - 1]
+    return [((t // nt) * 256, (t % nt) * 256) for t in picks]
+
+
+def test_llama_prefill_whole_c_and_whole_shared_tiles(hif4):
+    """Config 2 at M = 4096, default dispatch: the whole C against the single-CTA kernel entry by entry, and whole
+    256 x 256 tiles that two CTA pairs share (store, then reduce-add), plus the last tile, against the oracle."""
+    M = 4096
+    for (name, K, N) in wl.LLAMA3_8B_LINEARS:
+        w = hif4.hif4_quantize(wl.gaussian(N, K, 0.02, seed=2000 + N + K, device="cuda"))
+        x = hif4.hif4_quantize(wl.llama_activations(M, K, seed=1002 + M + K, device="cuda"))
+        C = hif4.hif4_gemm(x, w)
+        _whole_c_against_the_single_cta_kernel(hif4, x, w, C, f"llama {name} M={M}")
+        for (m0, n0) in _shared_tiles(M, N):
+            _tile_against_oracle(hif4, x, w, C, m0, n0, f"llama {name} M={M}")
+        _tile_against_oracle(hif4, x, w, C, M - 32, 0, f"llama {name} last rows", rows=32, cols=N)
+        del C, x, w
+        torch.cuda.empty_cache()
+
+
 def test_llama_linears_all_m(hif4):
     """Config 2 exactly as the benchmark runs it: every (M, K, N) through the default dispatch."""
     for (name, K, N) in wl.LLAMA3_8B_LINEARS:
@@ -115,6 +178,9 @@ def test_dense_prefill_m8192(hif4):
         w = hif4.hif4_quantize(wl.gaussian(N, K, 0.015, seed=4000 + N + K, device="cuda"))
         C = hif4.hif4_gemm(x, w)
         _sampled_entries(hif4, x, w, C, f"prefill {name}", n=300, seed=K)
+        _whole_c_against_the_single_cta_kernel(hif4, x, w, C, f"prefill {name}")
+        for (m0, n0) in _shared_tiles(wl.DENSE_PREFILL_M, N)[:2 if K > 8192 else 3]:
+            _tile_against_oracle(hif4, x, w, C, m0, n0, f"prefill {name}")
         del x, w, C
         torch.cuda.empty_cache()
 

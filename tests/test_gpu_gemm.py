@@ -177,11 +177,11 @@ def test_grouped_gemm_many_small_groups_wide_n(hif4):
     b = hif4.hif4_quantize((torch.randn(G * N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16)).view(G, N, K // 64, 36)
     out = hif4.hif4_grouped_gemm(a, b, off)
     assert torch.equal(out, hif4.hif4_grouped_gemm(a, b, off)), "two runs differ"
-    hif4.hif4_set_gemm_path(2)
+    hif4.hif4_debug_set_gemm_path(2)
     try:
         ref1 = hif4.hif4_grouped_gemm(a, b, off)
     finally:
-        hif4.hif4_set_gemm_path(0)
+        hif4.hif4_debug_set_gemm_path(0)
     assert (out - ref1).abs().max().item() <= 1e-5 * K * ref1.abs().max().item()
     off_h = off.cpu().numpy()
     for gsel in (0, 7, 60, 61, G - 1):
@@ -195,9 +195,9 @@ def test_grouped_gemm_many_small_groups_wide_n(hif4):
 @pytest.fixture(params=[2, 3], ids=["one_cta", "cta_pair"])
 def tc_path(hif4, request):
     """2 = single-CTA 128 x 256 kernel, 3 = CTA-pair 256 x 256 kernel, forced whatever the shape."""
-    hif4.hif4_set_gemm_path(request.param)
+    hif4.hif4_debug_set_gemm_path(request.param)
     yield hif4
-    hif4.hif4_set_gemm_path(0)
+    hif4.hif4_debug_set_gemm_path(0)
     assert hif4.hif4_last_device_status() == 0, "a bounded wait inside the kernel ran out"
 
 
@@ -240,7 +240,7 @@ def test_tensor_core_kernel_random_units_nan_and_guard_bands(tc_path):
 def test_cta_pair_kernel_few_columns_in_the_last_tile_repeated(hif4):
     """A last column tile with 8 valid columns leaves 15 of its 16 staged slabs unused; the staging
     buffers of the TMA-store epilogue must not be reused while a store still reads them."""
-    hif4.hif4_set_gemm_path(3)
+    hif4.hif4_debug_set_gemm_path(3)
     try:
         for (M, N, K) in [(300, 520, 1024), (257, 264, 256), (512, 1032, 512)]:
             g = torch.Generator(device="cuda"); g.manual_seed(M + N + K)
@@ -250,7 +250,7 @@ def test_cta_pair_kernel_few_columns_in_the_last_tile_repeated(hif4):
             for _ in range(20):
                 assert torch.equal(C, hif4.hif4_gemm(a, b)), "runs differ"
     finally:
-        hif4.hif4_set_gemm_path(0)
+        hif4.hif4_debug_set_gemm_path(0)
     assert hif4.hif4_last_device_status() == 0
 
 
@@ -270,11 +270,11 @@ def test_cta_pair_kernel_k_sliced_last_round(hif4, M, N, K):
     C = check_sampled(hif4, a, b, f"k-sliced {M}x{N}x{K}", n=1500, seed=K, C=hif4.hif4_gemm(a, b, out=out[1:M + 1, :N]))
     assert (out[0] == -3.0).all() and (out[M + 1] == -3.0).all() and (out[:, N:] == -3.0).all()
     # every entry of the tail tiles against the kernel that never slices (different FP32 summation order)
-    hif4.hif4_set_gemm_path(2)
+    hif4.hif4_debug_set_gemm_path(2)
     try:
         C1 = hif4.hif4_gemm(a, b)
     finally:
-        hif4.hif4_set_gemm_path(0)
+        hif4.hif4_debug_set_gemm_path(0)
     scale = (C1.abs().max() + 1e-30).item()
     assert (C.contiguous() - C1).abs().max().item() <= 1e-5 * scale * K
     for _ in range(3):
@@ -297,11 +297,11 @@ def test_cta_pair_kernel_random_shapes_against_the_single_cta_kernel(hif4):
         a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
         b = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
         C = check_sampled(hif4, a, b, f"random shape {M}x{N}x{K}", n=300, seed=M + N)
-        hif4.hif4_set_gemm_path(2)
+        hif4.hif4_debug_set_gemm_path(2)
         try:
             C1 = hif4.hif4_gemm(a, b)
         finally:
-            hif4.hif4_set_gemm_path(0)
+            hif4.hif4_debug_set_gemm_path(0)
         scale = (C1.abs().max() + 1e-30).item()
         assert (C - C1).abs().max().item() <= 1e-5 * scale * K, (M, N, K)
     assert hif4.hif4_last_device_status() == 0
@@ -340,9 +340,9 @@ def test_tensor_core_prefill_shape_sampled(tc_path):
 # ------------------------------------------------------------------ weight-streaming kernel (M <= 16)
 @pytest.fixture()
 def gemv_path(hif4):
-    hif4.hif4_set_gemm_path(4)
+    hif4.hif4_debug_set_gemm_path(4)
     yield hif4
-    hif4.hif4_set_gemm_path(0)
+    hif4.hif4_debug_set_gemm_path(0)
     assert hif4.hif4_last_device_status() == 0, "a bounded wait inside the kernel ran out"
 
 
@@ -434,7 +434,7 @@ def test_every_code_under_every_scale_passes_through_the_gemm_exactly(hif4, path
     Bh = _one_hot_units(K)
     want_all = oracle.dequantize(A_all, oracle.FP32)
     assert np.array_equal(oracle.dequantize(Bh, oracle.FP32), np.eye(K, dtype=np.float32))
-    hif4.hif4_set_gemm_path(path)
+    hif4.hif4_debug_set_gemm_path(path)
     try:
         for start in range(0, A_all.shape[0], rows):
             A = A_all[start:start + rows]
@@ -448,7 +448,7 @@ def test_every_code_under_every_scale_passes_through_the_gemm_exactly(hif4, path
             got_t = hif4.hif4_gemm(b, a).cpu().numpy()                     # and as the B operand
             assert np.array_equal(np.abs(got_t.T), np.abs(want_all[start:start + rows]))
     finally:
-        hif4.hif4_set_gemm_path(0)
+        hif4.hif4_debug_set_gemm_path(0)
     assert hif4.hif4_last_device_status() == 0
 
 
@@ -491,3 +491,54 @@ def test_linear_with_few_rows_quantizes_inside_the_token_preparation(hif4, M, N,
     want = hif4.hif4_gemm(hif4.hif4_quantize(x, mode), w)
     assert torch.equal(y.view(torch.int32), want.view(torch.int32)), "fused token preparation differs from quantize + GEMM"
     assert hif4.hif4_last_device_status() == 0
+
+
+# ------------------------------------------------------------------ failure reporting
+def test_a_bounded_wait_that_runs_out_is_reported_once_and_the_context_stays_usable(hif4):
+    """A kernel waits, with the library's bounded-wait helper and a 1 ms budget, on an mbarrier that nobody arrives
+    on (no copy or MMA in flight).  It gives up, raises the device error word and returns; the host reads
+    HIF4_ERR_DEVICE_TIMEOUT (7) once, then HIF4_OK, and the next GEMM on the same context is correct."""
+    assert hif4.hif4_last_device_status() == 0
+    hif4.hif4_debug_wait_timeout(1_000_000)
+    assert hif4.hif4_last_device_status() == 7
+    assert hif4.status_string(7)
+    assert hif4.hif4_last_device_status() == 0
+    with pytest.raises(hif4.Hif4Error) as ei:
+        hif4.hif4_debug_wait_timeout(10 ** 10)              # budgets beyond 0.1 s are refused, nothing is launched
+    assert ei.value.code == 2
+    x, w = wl.single_layer(device="cuda")
+    check_full(hif4, hif4.hif4_quantize(x), hif4.hif4_quantize(w), "gemm after a reported timeout")
+    assert hif4.hif4_last_device_status() == 0
+
+
+def test_gemm_workspace_is_valid_under_every_path_override(hif4):
+    """hif4_gemm_workspace reports one figure per shape that is enough whichever kernel the override selects."""
+    g = torch.Generator(device="cuda"); g.manual_seed(77)
+    try:
+        for (M, N, K) in ((8, 520, 512), (100, 700, 1024), (300, 300, 2048)):
+            a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
+            b = hif4.hif4_quantize(torch.randn(N, K, generator=g, device="cuda").to(torch.bfloat16))
+            hif4.hif4_debug_set_gemm_path(0)
+            need = hif4.hif4_gemm_workspace(M, N, K)
+            ws = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
+            ref, refabs = oracle.gemm_f64(a.cpu().numpy(), b.cpu().numpy(), nthreads=8)
+            for path in (0, 1, 2, 3, 4):
+                hif4.hif4_debug_set_gemm_path(path)
+                assert hif4.hif4_gemm_workspace(M, N, K) == need
+                c = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+                rc = hif4.lib.hif4_gemm(a.data_ptr(), b.data_ptr(), c.data_ptr(), M, N, K, N, ws.data_ptr(), need, None)
+                assert rc == 0, (M, N, K, path, rc)
+                err = np.abs(c.cpu().numpy().astype(np.float64) - ref)
+                assert np.all(err <= TOL * refabs + 1e-300), (M, N, K, path)
+    finally:
+        hif4.hif4_debug_set_gemm_path(0)
+
+
+def test_grouped_gemm_refuses_row_counts_beyond_its_tile_table(hif4):
+    off = torch.zeros(2, dtype=torch.int64, device="cuda")
+    before = hif4.launch_count()
+    rc = hif4.lib.hif4_grouped_gemm(off.data_ptr(), off.data_ptr(), off.data_ptr(), off.data_ptr(), 1, 2 ** 31, 64, 256, 64,
+                                    None, 0, None)
+    assert rc == 2 and hif4.launch_count() == before
+    with pytest.raises(hif4.Hif4Error):
+        hif4.hif4_grouped_gemm_workspace(1, 2 ** 31, 64, 256)

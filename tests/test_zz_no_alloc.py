@@ -1,8 +1,8 @@
 """hif4_grouped_gemm_noalloc through the C ABI: the grouped GEMM for callers that cannot allocate device
 memory (fixed memory plans, plug-ins without an allocator, sections where a cudaMalloc's device-wide
 synchronisation is not acceptable).  Its tile table sits in a fixed array inside the library, so this
-file checks that (a) it gives what hif4_grouped_gemm gives, on two calls in a row that reuse the array
-with different group layouts, (b) problems that do not fit the array are refused, nothing launched.
+file checks that (a) it gives what hif4_grouped_gemm gives and what the CPU oracle's FP64 product gives, within
+the GEMM tolerance, on two calls in a row that reuse the array with different group layouts, (b) problems that do not fit the array are refused, nothing launched.
 
 Collected last on purpose (file name): if it fails, a run that stops at the first failure has already
 run every other test."""
@@ -40,9 +40,16 @@ def _check_against_existing_entry_point(hif4, a, b, off, what):
     got = torch.full((total, N), -7.0, dtype=torch.float32, device="cuda")
     hif4.hif4_grouped_gemm_noalloc(a, b, off, out=got)             # built-in scratch
     torch.cuda.synchronize()
-    _, refabs = oracle.grouped_gemm_f64(a.cpu().numpy(), b.cpu().numpy(), off.cpu().numpy(), nthreads=8)
-    err = np.abs(got.cpu().numpy().astype(np.float64) - want.cpu().numpy().astype(np.float64))
-    assert np.all(err <= TOL * refabs + 1e-300), f"{what}: worst ratio {np.max(err / np.maximum(TOL * refabs, 1e-300)):.3g}"
+    ref, refabs = oracle.grouped_gemm_f64(a.cpu().numpy(), b.cpu().numpy(), off.cpu().numpy(), nthreads=8)
+    got64, want64 = got.cpu().numpy().astype(np.float64), want.cpu().numpy().astype(np.float64)
+    bound = TOL * refabs + 1e-300
+    # each entry point against the oracle's FP64 result (an error common to both kernels would show here) ...
+    for name, c in (("no-alloc", got64), ("workspace", want64)):
+        err = np.abs(c - ref)
+        assert np.all(err <= bound), f"{what}, {name} entry point vs oracle: worst ratio {np.max(err / bound):.3g}"
+    # ... and against each other (they run different kernels, so the bits may differ; the tolerance may not)
+    err = np.abs(got64 - want64)
+    assert np.all(err <= bound), f"{what}: worst ratio between the entry points {np.max(err / bound):.3g}"
 
 
 def test_two_calls_in_a_row_match_the_workspace_entry_point(hif4):
