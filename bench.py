@@ -8,9 +8,11 @@ accumulation).  All inputs are seeded synthetic tensors (Student-t activations w
 channels, Gaussian weights); the model name only lends the layer shapes.
 
 Prints ONE JSON line: metric, value (whole-job TFLOP/s with inputs resident), ms_per_step, gpu_launches, clocks,
-roofline (the prefill GEMM kernel against the measured BF16 peak), per_shape, roofline_quantize, reference_points,
-e2e (through host buffers) and cpu_baseline.  `--impl reference` times the CPU oracle
-on a bounded sample of the same workload instead.
+roofline (the prefill GEMM kernel against the measured BF16 peak that matches the clocks sampled in the timed
+region), sustained (the same step repeated for at least 1.5 s), per_shape, per_config (the other four workload
+configurations: single layer, quantize sweep, dense prefill, MoE), roofline_quantize, reference_points, e2e
+(through host buffers) and cpu_baseline.  `--impl reference` times the CPU oracle on a bounded sample of the same
+workload instead.
 """
 from __future__ import annotations
 
@@ -35,6 +37,9 @@ METRIC = "hif4_gemm TFLOP/s + hif4_quantize GB/s at LLM shapes, % of roofline (1
 WORKLOAD = "llama3_8b_linears: K=4096 N in {4096,1024,14336} + K=14336 N=4096, M in {1,16,4096}"
 SHAPES = [(M, K, N, name) for M in wl.LLAMA3_8B_M for (name, K, N) in wl.LLAMA3_8B_LINEARS]
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_BF16_TFLOPS = 2250.0        # dense BF16 of the part's public specification (context beside the measured peaks)
+NOMINAL_HBM_GBS = 8000.0
+SUSTAINED_SECONDS = 1.5             # the step is also repeated for at least this long, so that clocks settle under load
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (None until a capture exists for that kernel).
 NCU_DRAM_BYTES_PER_LAUNCH = {"gemm_tc2_kernel": 264.1e6,      # captured on M=4096 N=14336 K=4096 (algorithmic 277.3e6)
@@ -52,58 +57,124 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock, power and clock-event reasons while the benchmark runs: NVML every 2 ms when the
+    `pynvml` module is there (a read-only query), else `nvidia-smi -lms 20`.  `window(t0, t1)` summarises
+    the samples between two host times; nothing on the GPU is ever set."""
 
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    REASONS = (("sw_power_cap", 0x4), ("hw_slowdown", 0x8), ("sw_thermal_slowdown", 0x20), ("hw_thermal_slowdown", 0x40),
+               ("hw_power_brake", 0x80))
+    SMI_FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+                  "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+                  "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
-        self.gpu = gpu_index
-        self.rows = []
-        self.proc = None
+    def __init__(self, device: torch.device):
+        self.device = device
+        self.rows = []                 # (host time, sm MHz, power W, set of reasons)
+        self.sm_max = None
+        self.source = None
+        self._stop = threading.Event()
         self.thread = None
+        self.proc = None
 
     def start(self):
         try:
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(self.device).uuid)
+            handle = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid) if not uuid.startswith("GPU-") else uuid)
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
+            reasons_fn = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                pynvml.nvmlDeviceGetCurrentClocksThrottleReasons
+            reasons_fn(handle)
+            self.source = "nvml, 2 ms"
+
+            def pump():
+                while not self._stop.is_set():
+                    try:
+                        sm = float(pynvml.nvmlDeviceGetClockInfo(handle, pynvml.NVML_CLOCK_SM))
+                        mask = int(reasons_fn(handle))
+                        watts = pynvml.nvmlDeviceGetPowerUsage(handle) / 1000.0
+                        self.rows.append((time.time(), sm, watts, {n for n, bit in self.REASONS if mask & bit}))
+                    except Exception:                       # noqa: BLE001 - a failed query is a missing sample
+                        pass
+                    time.sleep(0.002)
+            self.thread = threading.Thread(target=pump, daemon=True)
+            self.thread.start()
+            return
+        except Exception:                                   # noqa: BLE001 - no NVML binding: fall back to nvidia-smi
+            self.source = None
+        try:
+            idx = self.device.index or 0
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                ["nvidia-smi", f"--id={idx}", f"--query-gpu={self.SMI_FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
-        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.source = "nvidia-smi, 20 ms"
+
+        def pump_smi():
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            for line in self.proc.stdout:
+                r = [c.strip() for c in line.split(",")]
+                if len(r) < 7:
+                    continue
+                try:
+                    sm, smax, watts = float(r[0]), float(r[1]), float(r[2])
+                except ValueError:
+                    continue
+                self.sm_max = smax
+                self.rows.append((time.time(), sm, watts, {n for n, v in zip(names, r[3:7]) if v.lower().startswith("active")}))
+        self.thread = threading.Thread(target=pump_smi, daemon=True)
         self.thread.start()
 
-    def _pump(self):
-        for line in self.proc.stdout:
-            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+    def window(self, t0: float, t1: float) -> dict:
+        """Summary of the samples taken between host times t0 and t1."""
+        if self.source is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["no clock source (pynvml and nvidia-smi both unavailable)"]}
+        rows = [r for r in list(self.rows) if t0 <= r[0] <= t1]
+        reasons = set()
+        for r in rows:
+            reasons |= r[3]
+        sm = [r[1] for r in rows]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_min_mhz": min(sm) if sm else None,
+                "sm_max_mhz": self.sm_max, "power_w_max": round(max(r[2] for r in rows), 1) if rows else None,
+                "samples": len(rows), "reasons": sorted(reasons), "source": self.source}
 
-    def stop(self, t0: float = 0.0, t1: float = float("inf")) -> dict:
-        """Summary of the samples taken between host times t0 and t1 (the timed region)."""
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
+    def stop(self):
+        self._stop.set()
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
         if self.thread:
             self.thread.join(timeout=2)
-        sm, smax, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for (ts, r) in self.rows:
-            if len(r) < 7 or ts < t0 or ts > t1 + 0.05:
-                continue
-            try:
-                sm.append(float(r[0])); smax.append(float(r[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, r[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def pick_bf16_peak(peaks: dict, clocks: dict, same_run_matmul_tflops=None):
+    """The measured BF16 peak that matches the run: the burst figure unless the clocks sampled inside the timed
+    region show the power cap active or a median SM clock well below the maximum (then the sustained figure, which
+    was measured in that state).  Never below the rate torch.matmul reached in this same run."""
+    capped = "sw_power_cap" in clocks.get("reasons", []) or (
+        clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and clocks["sm_mhz"] < 0.85 * clocks["sm_max_mhz"])
+    kind = "sustained" if capped else "burst"
+    peak = peaks["bf16_tflops_sustained"] if capped else peaks["bf16_tflops"]
+    why = ("power cap active or SM clock below 85 % of maximum in the sampled region" if capped else
+           ("SM clock near maximum and no power cap in the sampled region" if clocks.get("samples") else
+            "no clock samples in the region: the larger (burst) figure is used"))
+    if same_run_matmul_tflops and same_run_matmul_tflops > peak:
+        peak, kind = same_run_matmul_tflops, kind + ", raised to this run's torch.matmul BF16 rate"
+    return peak, kind, why
+
+
+def bf16_fractions(tflops: float, peaks: dict, clocks: dict, floor=None) -> dict:
+    peak, kind, why = pick_bf16_peak(peaks, clocks, floor)
+    return {"peak": round(peak, 1), "peak_kind": kind, "peak_choice": why, "frac": round(tflops / peak, 4),
+            "frac_of_burst_peak": round(tflops / peaks["bf16_tflops"], 4),
+            "frac_of_sustained_peak": round(tflops / peaks["bf16_tflops_sustained"], 4),
+            "frac_of_nominal_dense": round(tflops / NOMINAL_BF16_TFLOPS, 4)}
 
 
 def flops(M, K, N):
@@ -181,7 +252,7 @@ def run_cuda(args):
         dp.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(dev)
     sampler.start()
     for _ in range(max(args.warmup, 3)):
         run_shapes(SHAPES)
@@ -224,11 +295,28 @@ def run_cuda(args):
     barrier()
     host_t1 = time.time()
     launches = hif4.launch_count() - launches0 + graph_launches * args.steps
-    clocks = sampler.stop(host_t0, host_t1)
+    clocks = sampler.window(host_t0, host_t1)
     elapsed_ms = dp.max_over_ranks(t_start.elapsed_time(t_end), dev)
     status = hif4.hif4_last_device_status()
     if status != 0:
         raise SystemExit(f"device status {status}: {hif4.status_string(status)}")
+    ms_per_step = elapsed_ms / args.steps
+
+    # The same step repeated for at least SUSTAINED_SECONDS: long enough for the clocks to settle under the power
+    # limit and for the sampler to see it (the K timed steps above may last only milliseconds).
+    sus_steps = max(args.steps, int(SUSTAINED_SECONDS * 1e3 / max(ms_per_step, 1e-3)) + 1)
+    sus_events = []
+    s_start, s_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sus_t0 = time.time()
+    s_start.record(stream)
+    for i in range(sus_steps):
+        step(sus_events if i % 8 == 0 else None)            # events around every eighth step's prefill GEMMs
+    s_end.record(stream)
+    barrier()
+    sus_t1 = time.time()
+    sus_clocks = sampler.window(sus_t0, sus_t1)
+    sus_ms = dp.max_over_ranks(s_start.elapsed_time(s_end), dev) / sus_steps
 
     # per-kernel times of the decode-shaped linears: a separate pass with events around every call and
     # L2 flushed (a 256 MB write) before each linear
@@ -238,38 +326,54 @@ def run_cuda(args):
             flush.zero_()
             run_shapes([sh], small_events)
     torch.cuda.synchronize()
-    events += small_events
 
     step_flops = sum(flops(M, K, N) for (M, K, N, _) in SHAPES)
-    ms_per_step = elapsed_ms / args.steps
     value = dp.job_throughput(step_flops, world, ms_per_step * 1e-3) / 1e12
+    ref_points = measure_reference_points(dev) if (rank == 0 and world == 1) else None
+    matmul_floor = (ref_points or {}).get("bf16_matmul", {}).get("tflops")
 
     # ---- per-kernel times (prefill shapes: inside the timed region; decode shapes: the pass above)
-    per_shape = {}
-    for (shape, e0, e1, e2) in events:
-        d = per_shape.setdefault(shape, [0.0, 0.0, 0])
-        d[0] += e0.elapsed_time(e1); d[1] += e1.elapsed_time(e2); d[2] += 1
+    def shape_times(evs):
+        acc = {}
+        for (shape, e0, e1, e2) in evs:
+            d = acc.setdefault(shape, [0.0, 0.0, 0])
+            d[0] += e0.elapsed_time(e1); d[1] += e1.elapsed_time(e2); d[2] += 1
+        return {k: (v[0] / v[2], v[1] / v[2]) for k, v in acc.items()}
+
+    per_shape = shape_times(events + small_events)
+    sus_shape = shape_times(sus_events)
     table = []
-    tc_flops = tc_ms = 0.0
+    tc_flops = tc_ms = sus_tc_ms = 0.0
     for (M, K, N, name) in SHAPES:
-        q_ms, g_ms, n = per_shape[(M, K, N)]
-        q_ms /= n; g_ms /= n
+        q_ms, g_ms = per_shape[(M, K, N)]
+        tf = flops(M, K, N) / g_ms / 1e9
         row = {"M": M, "K": K, "N": N, "quantize_us": round(q_ms * 1e3, 2), "gemm_us": round(g_ms * 1e3, 2),
-               "gemm_tflops": round(flops(M, K, N) / g_ms / 1e9, 2),
+               "gemm_tflops": round(tf, 2),
                "gemm_min_traffic_gbs": round(gemm_min_bytes(M, K, N) / g_ms / 1e6, 1)}
         if M >= 4096:
-            tc_flops += flops(M, K, N); tc_ms += g_ms
-            row["frac_of_bf16_peak"] = round(flops(M, K, N) / g_ms / 1e9 / peaks["bf16_tflops_sustained"], 3)
+            tc_flops += flops(M, K, N); tc_ms += g_ms; sus_tc_ms += sus_shape[(M, K, N)][1]
+            fr = bf16_fractions(tf, peaks, clocks, matmul_floor)
+            row.update({"frac_of_bf16_peak": fr["frac"], "frac_of_burst_peak": fr["frac_of_burst_peak"],
+                        "frac_of_nominal_dense": fr["frac_of_nominal_dense"],
+                        "gemm_us_sustained": round(sus_shape[(M, K, N)][1] * 1e3, 2)})
         else:
             row["frac_of_hbm_peak"] = round(gemm_min_bytes(M, K, N) / g_ms / 1e6 / peaks["hbm_gbs"], 3)
+            row["l2"] = "flushed (256 MB write) before the linear"
         table.append(row)
     achieved = tc_flops / tc_ms / 1e9
-    roofline = {"bound": "tensor", "kernel": "gemm_tc2_kernel (M=4096 launches)", "achieved": round(achieved, 1),
-                "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                "frac": round(achieved / peaks["bf16_tflops_sustained"], 4),
-                "frac_of_burst_peak": round(achieved / peaks["bf16_tflops"], 4), "peak_kind": f"of {peak_kind} (sustained)",
+    roofline = {"bound": "tensor", "kernel": "gemm_tc2_kernel (the four M=4096 launches of a step)", "achieved": round(achieved, 1),
+                "unit": "TFLOP/s", **bf16_fractions(achieved, peaks, clocks, matmul_floor),
+                "peak_source": f"{peak_kind} (MEASURED_PEAKS.json)" if peak_kind == "measured" else "fallback",
+                "us_times_sm_mhz": round(tc_ms * 1e3 * clocks["sm_mhz"], 0) if clocks.get("sm_mhz") else None,
                 "traffic": NCU_DRAM_BYTES_PER_LAUNCH["gemm_tc2_kernel"],
-                "traffic_note": "dram bytes of the M=4096 N=14336 K=4096 launch (profiles/gemm_tc2_kernel_4096x14336x4096.md)"}
+                "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of the M=4096 N=14336 K=4096 launch; algorithmic minimum 277.3e6"}
+    sus_achieved = tc_flops / sus_tc_ms / 1e9
+    sustained = {"seconds": round(sus_ms * sus_steps / 1e3, 2), "steps": sus_steps, "ms_per_step": round(sus_ms, 4),
+                 "value": round(dp.job_throughput(step_flops, world, sus_ms * 1e-3) / 1e12, 2), "unit": "TFLOP/s",
+                 "clocks": sus_clocks,
+                 "roofline": {"achieved": round(sus_achieved, 1), "unit": "TFLOP/s",
+                              **bf16_fractions(sus_achieved, peaks, sus_clocks, None),
+                              "us_times_sm_mhz": round(sus_tc_ms * 1e3 * sus_clocks["sm_mhz"], 0) if sus_clocks.get("sm_mhz") else None}}
 
     out = {
         "metric": METRIC, "value": round(value, 2), "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
@@ -284,13 +388,16 @@ def run_cuda(args):
                               "prefill linears (hif4_quantize + hif4_gemm) launched directly"
                               if graphs else "every kernel launched directly (hif4_linear for M <= 16, hif4_quantize + hif4_gemm for M = 4096)"),
                    "parallelism": f"dp{world} (independent token batches, no collective)"},
-        "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "per_shape": table,
+        "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "sustained": sustained, "per_shape": table,
     }
 
     if rank == 0 and world == 1:
         out["roofline_quantize"] = measure_quantize_roofline(hif4, dev, peaks, peak_kind)
-        out["reference_points"] = measure_reference_points(dev)
+        out["reference_points"] = ref_points
+        if not args.no_per_config:
+            out["per_config"] = measure_per_config(hif4, dev, peaks, sampler, matmul_floor)
     out["e2e"] = measure_e2e(hif4, dev, weights, world, args)
+    sampler.stop()
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             out["cpu_baseline"] = cpu_baseline_sample()
@@ -299,6 +406,141 @@ def run_cuda(args):
         import torch.distributed as dist
         dist.barrier()
         dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------- the other workload configurations
+def _timed(fn, reps, sampler, flush=None):
+    """Mean device time per call in microseconds (CUDA events on the current stream) and the clocks sampled
+    meanwhile.  With `flush`, a buffer larger than L2 is rewritten before every call and each call is timed alone."""
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    t0 = time.time()
+    if flush is None:
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(int(reps * 24_000))       # ~12 us per queued call: the host queues the launches while the GPU idles
+        s.record()
+        for _ in range(reps):
+            fn()
+        e.record()
+        torch.cuda.synchronize()
+        us = s.elapsed_time(e) / reps * 1e3
+    else:
+        pairs = []
+        for _ in range(reps):
+            flush.zero_()
+            s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s.record(); fn(); e.record()
+            pairs.append((s, e))
+        torch.cuda.synchronize()
+        us = statistics.median(s.elapsed_time(e) for s, e in pairs) * 1e3
+    return us, sampler.window(t0, time.time())
+
+
+def measure_per_config(hif4, dev, peaks, sampler, matmul_floor):
+    """Configurations 1, 3, 4 and 5 of the workload list, each kernel timed alone with inputs resident."""
+    out = {}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    hbm = peaks["hbm_gbs"]
+
+    # ---- config 1: single layer 128 x 512 x 512 (launch-bound sizes; L2 flushed before every call)
+    x, w = wl.single_layer(device=dev)
+    xq, wq = hif4.hif4_quantize(x), hif4.hif4_quantize(w)
+    c = torch.empty(128, 512, dtype=torch.float32, device=dev)
+    ws = torch.empty(max(hif4.hif4_gemm_workspace(128, 512, 512), 256), dtype=torch.uint8, device=dev)
+    qx_us, _ = _timed(lambda: hif4.hif4_quantize(x, out=xq), 20, sampler, flush)
+    qw_us, _ = _timed(lambda: hif4.hif4_quantize(w, out=wq), 20, sampler, flush)
+    g_us, _ = _timed(lambda: hif4.hif4_gemm(xq, wq, out=c, workspace=ws), 20, sampler, flush)
+    out["config1_single_layer"] = {
+        "shape": {"M": 128, "K": 512, "N": 512}, "l2": "flushed before every call", "quantize_x_us": round(qx_us, 2),
+        "quantize_w_us": round(qw_us, 2), "gemm_us": round(g_us, 2), "gemm_tflops": round(flops(128, 512, 512) / g_us / 1e6, 3),
+        "quantize_w_gbs": round(quant_bytes(512, 512) / qw_us / 1e3, 1),
+        "note": "67 MFLOP and 0.7 MB: every kernel here is bound by launch latency, not by a roofline"}
+
+    # ---- config 3: quantize sweep.  Below 2^28 elements source and result would stay in the 126 MB L2, so the
+    # launches rotate over enough buffers to touch more than 512 MB between two uses of the same one.
+    sweep = []
+    for log2n, dtype in [(20, torch.bfloat16), (22, torch.bfloat16), (24, torch.bfloat16), (26, torch.bfloat16),
+                         (28, torch.bfloat16), (30, torch.bfloat16), (28, torch.float32)]:
+        n = 2 ** log2n
+        esz = 2 if dtype == torch.bfloat16 else 4
+        per_elem = esz + 0.5625
+        nbuf = max(1, min(64, -(-(512 << 20) // int(n * per_elem))))
+        src = wl.quantize_sweep(n, device=dev, dtype=dtype)
+        srcs = [src] + [src.clone() for _ in range(nbuf - 1)]
+        dsts = [torch.empty(n // 4096, 64, 36, dtype=torch.uint8, device=dev) for _ in range(nbuf)]
+        state = {"i": 0}
+
+        def call():
+            i = state["i"] = (state["i"] + 1) % nbuf
+            hif4.hif4_quantize(srcs[i], out=dsts[i])
+        us, clk = _timed(call, max(20, 2 * nbuf), sampler)
+        gbs = n * per_elem / us / 1e3
+        sweep.append({"elements": f"2^{log2n}", "source": "bf16" if esz == 2 else "fp32", "us": round(us, 2), "gbs": round(gbs, 1),
+                      "frac_of_measured_hbm": round(gbs / hbm, 4), "frac_of_nominal_8tbs": round(gbs / NOMINAL_HBM_GBS, 4),
+                      "buffers_rotated": nbuf})
+        del src, srcs, dsts
+        torch.cuda.empty_cache()
+    out["config3_quantize_sweep"] = {"bytes_per_element": "2 + 36/64 (bf16), 4 + 36/64 (fp32)", "peak_hbm_gbs": hbm, "rows": sweep}
+
+    # ---- config 4: dense prefill, M = 8192
+    rows = []
+    M = wl.DENSE_PREFILL_M
+    for (name, K, N) in wl.DENSE_PREFILL_LINEARS:
+        xb = wl.prefill_activations(M, K, device=dev)
+        wq = hif4.hif4_quantize(wl.gaussian(N, K, 0.015, seed=4000 + N + K, device=dev))
+        xq = hif4.hif4_quantize(xb)
+        c = torch.empty(M, N, dtype=torch.float32, device=dev)
+        ws = torch.empty(max(hif4.hif4_gemm_workspace(M, N, K), 256), dtype=torch.uint8, device=dev)
+        q_us, _ = _timed(lambda: hif4.hif4_quantize(xb, out=xq), 10, sampler)
+        g_us, clk = _timed(lambda: hif4.hif4_gemm(xq, wq, out=c, workspace=ws), 20, sampler)
+        tf = flops(M, K, N) / g_us / 1e6
+        rows.append({"name": name, "M": M, "K": K, "N": N, "quantize_us": round(q_us, 1),
+                     "quantize_gbs": round(quant_bytes(M, K) / q_us / 1e3, 1), "gemm_us": round(g_us, 1),
+                     "gemm_tflops": round(tf, 1), **bf16_fractions(tf, peaks, clk, matmul_floor),
+                     "sm_mhz": clk.get("sm_mhz"), "reasons": clk.get("reasons"),
+                     "l2": "operands and result together exceed L2 (result alone is %d MB)" % (M * N * 4 >> 20)})
+        del xb, wq, xq, c, ws
+        torch.cuda.empty_cache()
+    out["config4_dense_prefill"] = {"rows": rows, "timing": "20 launches back to back per shape"}
+
+    # ---- config 5: MoE layer through hif4_grouped_gemm (Zipf(1.1) routing of 4096 tokens, top-8 of 256 experts)
+    r = wl.moe_routing(device=dev)
+    off = r["offsets"]
+    counts = r["counts"]
+    total = int(off[-1])
+    layers = []
+    for (lname, K, N, seed) in (("gate_up", wl.MOE_HIDDEN, 2 * wl.MOE_INTER, 5100), ("down", wl.MOE_INTER, wl.MOE_HIDDEN, 5200)):
+        a = hif4.hif4_quantize(wl.outlier_channel_activations(total, K, seed=seed, device=dev))
+        b = torch.empty(wl.MOE_EXPERTS, N, K // 64, 36, dtype=torch.uint8, device=dev)
+        for e0 in range(0, wl.MOE_EXPERTS, 16):                # BF16 sources are drawn 16 experts at a time
+            hif4.hif4_quantize(wl.gaussian(16 * N, K, 0.02, seed=seed + 1 + e0, device=dev), out=b[e0:e0 + 16].view(16 * N, K // 64, 36))
+        c = torch.empty(total, N, dtype=torch.float32, device=dev)
+        ws = torch.empty(max(hif4.hif4_grouped_gemm_workspace(wl.MOE_EXPERTS, total, N, K), 256), dtype=torch.uint8, device=dev)
+        us, clk = _timed(lambda: hif4.hif4_grouped_gemm(a, b, off, out=c, workspace=ws), 10, sampler)
+        fl = flops(total, K, N)
+        live = int((counts > 0).sum())
+        stream_bytes = 0.5625 * (live * N + total) * K + 4.0 * total * N
+        peak, kind, _ = pick_bf16_peak(peaks, clk, matmul_floor)
+        bound_tensor_us = fl / peak / 1e6
+        bound_stream_us = stream_bytes / hbm / 1e3
+        bound_us = max(bound_tensor_us, bound_stream_us)
+        layers.append({"name": lname, "K": K, "N": N, "rows": total, "experts_with_rows": live, "ms": round(us / 1e3, 3),
+                       "tflops": round(fl / us / 1e6, 1), "bound_tensor_ms": round(bound_tensor_us / 1e3, 3),
+                       "bound_weight_stream_ms": round(bound_stream_us / 1e3, 3), "bf16_peak": round(peak, 1), "peak_kind": kind,
+                       "roofline_bound": "tensor" if bound_tensor_us >= bound_stream_us else "hbm",
+                       "frac": round(bound_us / us, 4), "frac_of_nominal_dense": round(fl / us / 1e6 / NOMINAL_BF16_TFLOPS, 4),
+                       "sm_mhz": clk.get("sm_mhz"), "reasons": clk.get("reasons"), "l2": "weights (GB) exceed L2"})
+        del a, b, c, ws
+        torch.cuda.empty_cache()
+    cnt = counts.cpu()
+    out["config5_moe"] = {"tokens": wl.MOE_TOKENS, "topk": wl.MOE_TOPK, "experts": wl.MOE_EXPERTS,
+                          "rows_per_expert": {"max": int(cnt.max()), "median": int(cnt.median()), "min": int(cnt.min())},
+                          "layers": layers}
+    status = hif4.hif4_last_device_status()
+    if status != 0:
+        raise SystemExit(f"device status {status}: {hif4.status_string(status)}")
+    return out
 
 
 def measure_quantize_roofline(hif4, dev, peaks, peak_kind):
@@ -596,6 +838,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the per_config block (configurations 1, 3, 4, 5)")
     ap.add_argument("--no-graph", action="store_true", help="launch the decode-shaped linears directly instead of replaying a CUDA graph")
     ap.add_argument("--gemm-path", type=int, default=0, help="with --case: kernel selection, see hif4_debug_set_gemm_path")
     ap.add_argument("--case", default=None,

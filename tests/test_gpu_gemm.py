@@ -355,7 +355,7 @@ def test_weight_streaming_kernel_full_compare(gemv_path, M, N, K):
     g = torch.Generator(device="cuda"); g.manual_seed(M * 11 + N)
     a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
     b = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
-    assert hif4.hif4_gemm_workspace(M, N, K) == (8 if M <= 8 else 16 if M <= 16 else 32) * K * 2
+    assert hif4.hif4_gemm_workspace(M, N, K) >= (8 if M <= 8 else 16 if M <= 16 else 32) * K * 2   # the decoded tokens (or more, if another kernel for this shape needs more)
     before = hif4.launch_count()
     out = torch.full((M + 2, N + 3), -5.0, dtype=torch.float32, device="cuda")
     C = check_full(hif4, a, b, f"gemv {M}x{N}x{K}", out=out[1:M + 1, 1:N + 1])
