@@ -537,6 +537,21 @@ def measure_per_config(hif4, dev, peaks, sampler, matmul_floor):
     out["config5_moe"] = {"tokens": wl.MOE_TOKENS, "topk": wl.MOE_TOPK, "experts": wl.MOE_EXPERTS,
                           "rows_per_expert": {"max": int(cnt.max()), "median": int(cnt.median()), "min": int(cnt.min())},
                           "layers": layers}
+    # ---- the quantization-error study of Section III-A (18 Gaussian 1024 x 1024 matrices, sigma = 0.01 * 2^x)
+    study = []
+    for xexp in range(18):
+        g = torch.Generator(device=dev); g.manual_seed(7000 + xexp)
+        x = (torch.randn(1024, 1024, generator=g, device=dev) * (0.01 * 2.0 ** xexp)).to(torch.bfloat16)
+        errs = [float(hif4.hif4_mse_roundtrip(x, fmt, want_image=False)[1].item()) for fmt in (0, 1, 2, 3)]
+        study.append({"x": xexp, "mse_hif4": errs[0] / x.numel(), "mxfp4": round(errs[1] / errs[0], 4),
+                      "nvfp4_direct": round(errs[2] / errs[0], 4), "nvfp4_pts": round(errs[3] / errs[0], 4)})
+    x = (torch.randn(1024, 1024, device=dev)).to(torch.bfloat16)
+    us = {name: round(_timed(lambda f=fmt: hif4.hif4_mse_roundtrip(x, f, want_image=False), 20, sampler)[0], 1)
+          for name, fmt in (("hif4", 0), ("mxfp4", 1), ("nvfp4", 2), ("nvfp4_pts", 3))}
+    out["mse_study"] = {"what": "MSE of each format divided by HiF4's, BF16 sources, computed by hif4_mse_roundtrip",
+                        "paper": "HiF4 : NVFP4 : MXFP4 = 1 : 1.32 : 1.89", "mean_nvfp4_pts": round(statistics.mean(r["nvfp4_pts"] for r in study), 4),
+                        "mean_mxfp4": round(statistics.mean(r["mxfp4"] for r in study), 4), "rows": study,
+                        "us_per_1024x1024_matrix": us}
     status = hif4.hif4_last_device_status()
     if status != 0:
         raise SystemExit(f"device status {status}: {hif4.status_string(status)}")

@@ -192,6 +192,23 @@ hif4_status hif4_grouped_gemm_noalloc(const void* A_units, const void* B_units, 
 /* Size in bytes of the built-in scratch array (HIF4_NOALLOC_SCRATCH_BYTES).  Host-only.  */
 size_t hif4_grouped_gemm_noalloc_capacity(void);
 
+/* hif4_mse_roundtrip -- the quantization-error experiment of Section III-A for one tensor: convert a BF16 tensor
+ * to a 4-bit block format and back, write the image as FP32 and sum the squared error against the source.
+ *   HIF4_FMT_HIF4       Algorithm 1 (round-half-to-even), then Eq. 2
+ *   HIF4_FMT_MXFP4      blocks of 32, power-of-two scale 2^(floor(log2 amax) - 2), E2M1 elements
+ *   HIF4_FMT_NVFP4      blocks of 16, E4M3 scale = amax / 6, E2M1 elements ("direct cast")
+ *   HIF4_FMT_NVFP4_PTS  NVFP4 after per-tensor scaling of the peak magnitude to 2688, undone afterwards
+ * (E2M1 and E4M3 rounding to nearest, ties to even, saturating; every step one FP32 operation.)
+ *   src_bf16    device, n BF16 elements, 16-byte aligned; n a multiple of 64.
+ *   dst         device, n FP32 elements receiving the image, or NULL when only the error is wanted.
+ *   sq_err_sum  device, one FP64: sum over the elements of (image - source)^2, accumulated in FP64 in an order
+ *               that does not depend on scheduling.
+ *   workspace   device scratch of at least hif4_mse_workspace bytes, 256-byte aligned.  */
+typedef enum { HIF4_FMT_HIF4 = 0, HIF4_FMT_MXFP4 = 1, HIF4_FMT_NVFP4 = 2, HIF4_FMT_NVFP4_PTS = 3 } hif4_bfp4_format;
+hif4_status hif4_mse_workspace(int64_t n, hif4_bfp4_format fmt, size_t* bytes);
+hif4_status hif4_mse_roundtrip(const void* src_bf16, int64_t n, hif4_bfp4_format fmt, float* dst, double* sq_err_sum,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream` and returns HIF4_ERR_DEVICE_TIMEOUT if any kernel of this library gave up
  * a bounded wait since the last call (the flag is cleared), HIF4_ERR_CUDA if the stream reports
  * an error, else HIF4_OK.  For tests and debugging.  */

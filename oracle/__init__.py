@@ -68,6 +68,17 @@ def lib() -> ctypes.CDLL:
         L.hif4_ref_best_unit.restype = dbl
         L.hif4_ref_best_unit.argtypes = [vp, vp]
         L.hif4_ref_hardware_threads.restype = ci
+        flt, fp = ctypes.c_float, ctypes.c_void_p
+        L.hif4_ref_e2m1_round.restype = flt
+        L.hif4_ref_e2m1_round.argtypes = [flt]
+        L.hif4_ref_e4m3_round.restype = flt
+        L.hif4_ref_e4m3_round.argtypes = [flt]
+        L.hif4_ref_pts_gain.restype = flt
+        L.hif4_ref_pts_gain.argtypes = [fp, i64]
+        L.hif4_ref_mxfp4_roundtrip.restype = ci
+        L.hif4_ref_mxfp4_roundtrip.argtypes = [fp, i64, fp]
+        L.hif4_ref_nvfp4_roundtrip.restype = ci
+        L.hif4_ref_nvfp4_roundtrip.argtypes = [fp, i64, flt, fp]
         _lib = L
     return _lib
 
@@ -194,6 +205,37 @@ def best_unit(x: np.ndarray):
     out = np.zeros(UNIT_BYTES, dtype=np.uint8)
     err = float(lib().hif4_ref_best_unit(_ptr(x), _ptr(out)))
     return err, out
+
+
+# ---- comparison formats of the quantization-error study (Section III-A)
+def e2m1_round(q: float) -> float:
+    return float(lib().hif4_ref_e2m1_round(float(q)))
+
+
+def e4m3_round(v: float) -> float:
+    return float(lib().hif4_ref_e4m3_round(float(v)))
+
+
+def pts_gain(x: np.ndarray) -> float:
+    """2688 / max|x| (one FP32 division): the per-tensor scaling that precedes NVFP4 in the study."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    return float(lib().hif4_ref_pts_gain(_ptr(x), x.size))
+
+
+def mxfp4_roundtrip(x: np.ndarray) -> np.ndarray:
+    """float32 array (size a multiple of 32) -> its MXFP4 quantize-dequantize image, float32."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty_like(x)
+    _check(lib().hif4_ref_mxfp4_roundtrip(_ptr(x), x.size, _ptr(out)), "mxfp4_roundtrip")
+    return out
+
+
+def nvfp4_roundtrip(x: np.ndarray, gain: float = 1.0) -> np.ndarray:
+    """float32 array (size a multiple of 16) -> its NVFP4 image; gain = pts_gain(x) applies per-tensor scaling."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty_like(x)
+    _check(lib().hif4_ref_nvfp4_roundtrip(_ptr(x), x.size, float(np.float32(gain)), _ptr(out)), "nvfp4_roundtrip")
+    return out
 
 
 # ---- small numpy conveniences for BF16 bit patterns (storage conversion only, no method arithmetic)

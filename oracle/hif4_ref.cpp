@@ -2,7 +2,8 @@
 //
 // TEST INFRASTRUCTURE ONLY.  This is a plain, slow, obviously-correct restatement of what the
 // paper defines: decode (Eq. 2), the BF16/FP32 -> HiF4 conversion (Algorithm 1, Section II-B),
-// the dot product (Eq. 3) and a flat FP64 GEMM on decoded values.  It shares no code, table or
+// the dot product (Eq. 3), a flat FP64 GEMM on decoded values, and the MXFP4 / NVFP4 round trips that the
+// quantization-error study of Section III-A compares HiF4 with.  It shares no code, table or
 // constant with the CUDA library and must never be linked into or called from it; only the test
 // suite, the smoke check and the benchmark's CPU-baseline leg use it.
 //
@@ -432,6 +433,84 @@ double hif4_ref_best_unit(const double* x, void* best_unit) {
   }
   if (best_unit) std::memcpy(best_unit, bestu, kUnitBytes);
   return best;
+}
+
+// ---------------------------------------------------------------- comparison formats of Section III-A
+// The quantization-error study converts the same matrices to MXFP4 and NVFP4 as well.  Both are published
+// formats; only what the study needs is restated here (quantize-then-dequantize of a flat array), in FP32
+// arithmetic with IEEE round-to-nearest-even operations, one operation per step, so that a GPU kernel can be
+// compared bit for bit.
+//   E2M1 element: magnitudes {0, 0.5, 1, 1.5, 2, 3, 4, 6}, round to nearest, ties to the even code, saturating.
+//   MXFP4: blocks of 32, power-of-two scale 2^(floor(log2 amax) - 2) (2 = the largest E2M1 exponent), exponent
+//          clamped to [-127, 127]; elements round(x / scale), so values between 6 and 8 scales saturate to 6.
+//   NVFP4: blocks of 16, scale = E4M3(amax / 6) ("normalize the peak magnitude of each group to 6"), elements
+//          round(x / scale).  With per-tensor scaling the tensor is first multiplied by gain = 2688 / max|x|
+//          (2688 = 448 * 6) and the result divided by the gain again.
+namespace {
+const float kE2M1[8] = {0.0f, 0.5f, 1.0f, 1.5f, 2.0f, 3.0f, 4.0f, 6.0f};
+
+float e2m1_round(float q) {                       // q >= 0
+  int best = 0;
+  for (int c = 1; c < 8; ++c) {
+    const float d_best = std::fabs(q - kE2M1[best]), d_c = std::fabs(q - kE2M1[c]);
+    if (d_c < d_best || (d_c == d_best && (c % 2 == 0))) best = c;     // nearest; a tie goes to the even code
+  }
+  return kE2M1[best];
+}
+
+// FP8 E4M3 (bias 7, 3 mantissa bits, subnormals in steps of 2^-9, largest value 448): nearest-even, saturating.
+float e4m3_round(float v) {                       // v >= 0, finite
+  if (v == 0.0f) return 0.0f;
+  int e = std::ilogb(v);
+  if (e < -6) e = -6;
+  const float quantum = std::ldexp(1.0f, e - 3);
+  const float r = std::nearbyint(v / quantum) * quantum;           // division by a power of two: exact
+  return r > 448.0f ? 448.0f : r;
+}
+}  // namespace
+
+float hif4_ref_e2m1_round(float q) { return e2m1_round(q); }
+float hif4_ref_e4m3_round(float v) { return e4m3_round(v); }
+
+// 2688 / max|x| in FP32 (one division); 1 for an all-zero tensor.
+float hif4_ref_pts_gain(const float* x, int64_t n) {
+  float amax = 0.0f;
+  for (int64_t i = 0; i < n; ++i) amax = std::max(amax, std::fabs(x[i]));
+  return amax > 0.0f ? 2688.0f / amax : 1.0f;
+}
+
+int hif4_ref_mxfp4_roundtrip(const float* x, int64_t n, float* out) {
+  if (!x || !out) return 1;
+  if (n < 0 || n % 32) return 2;
+  for (int64_t b = 0; b < n; b += 32) {
+    float amax = 0.0f;
+    for (int i = 0; i < 32; ++i) amax = std::max(amax, std::fabs(x[b + i]));
+    if (amax == 0.0f) { for (int i = 0; i < 32; ++i) out[b + i] = std::copysign(0.0f, x[b + i]); continue; }
+    int e = std::ilogb(amax) - 2;
+    e = std::min(127, std::max(-127, e));
+    const float scale = std::ldexp(1.0f, e);
+    for (int i = 0; i < 32; ++i) {
+      const float q = std::fabs(x[b + i]) / scale;
+      out[b + i] = std::copysign(e2m1_round(q) * scale, x[b + i]);
+    }
+  }
+  return 0;
+}
+
+int hif4_ref_nvfp4_roundtrip(const float* x, int64_t n, float gain, float* out) {
+  if (!x || !out) return 1;
+  if (n < 0 || n % 16) return 2;
+  for (int64_t b = 0; b < n; b += 16) {
+    float v[16], amax = 0.0f;
+    for (int i = 0; i < 16; ++i) { v[i] = x[b + i] * gain; amax = std::max(amax, std::fabs(v[i])); }
+    const float scale = e4m3_round(amax / 6.0f);
+    for (int i = 0; i < 16; ++i) {
+      float d = 0.0f;
+      if (scale > 0.0f) d = e2m1_round(std::fabs(v[i]) / scale) * scale;
+      out[b + i] = std::copysign(d, x[b + i]) / gain;
+    }
+  }
+  return 0;
 }
 
 int hif4_ref_hardware_threads(void) {

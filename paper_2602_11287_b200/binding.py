@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libhif4.so")
 UNIT_ELEMS, UNIT_BYTES = 64, 36
 HIF4_BF16, HIF4_FP32, HIF4_FP16 = 0, 1, 2
 HIF4_RNE, HIF4_RHA = 0, 1
+HIF4_FMT_HIF4, HIF4_FMT_MXFP4, HIF4_FMT_NVFP4, HIF4_FMT_NVFP4_PTS = 0, 1, 2, 3
 HIF4_OK = 0
 
 EXPORTED_SYMBOLS = [
@@ -25,6 +26,7 @@ EXPORTED_SYMBOLS = [
     "hif4_grouped_gemm_workspace", "hif4_grouped_gemm", "hif4_last_device_status", "hif4_status_string",
     "hif4_debug_launch_count", "hif4_debug_set_gemm_path", "hif4_grouped_gemm_noalloc", "hif4_grouped_gemm_noalloc_capacity",
     "hif4_linear", "hif4_linear_workspace", "hif4_quantize_transposed", "hif4_debug_wait_timeout",
+    "hif4_mse_workspace", "hif4_mse_roundtrip",
 ]
 
 
@@ -65,6 +67,10 @@ def _load() -> ctypes.CDLL:
     L.hif4_linear_workspace.argtypes = [i64, i64, i64, ctypes.POINTER(sz)]
     L.hif4_linear.restype = ci
     L.hif4_linear.argtypes = [vp, ci, i64, vp, vp, i64, i64, i64, i64, ci, vp, sz, vp]
+    L.hif4_mse_workspace.restype = ci
+    L.hif4_mse_workspace.argtypes = [i64, ci, ctypes.POINTER(sz)]
+    L.hif4_mse_roundtrip.restype = ci
+    L.hif4_mse_roundtrip.argtypes = [vp, i64, ci, vp, vp, vp, sz, vp]
     L.hif4_last_device_status.restype = ci
     L.hif4_last_device_status.argtypes = [vp]
     L.hif4_status_string.restype = ctypes.c_char_p
@@ -288,6 +294,29 @@ def hif4_debug_set_gemm_path(path: int) -> None:
     """Test hook: 0 = by shape, 1 = CUDA-core kernel, 2 = single-CTA tensor-core kernel, 3 = CTA-pair kernel,
     4 = weight-streaming kernel (each whenever legal)."""
     _check("hif4_debug_set_gemm_path", lib.hif4_debug_set_gemm_path(path))
+
+
+def hif4_mse_workspace(n: int, fmt: int) -> int:
+    b = ctypes.c_size_t(0)
+    _check("hif4_mse_workspace", lib.hif4_mse_workspace(n, fmt, ctypes.byref(b)))
+    return int(b.value)
+
+
+def hif4_mse_roundtrip(src: torch.Tensor, fmt: int, want_image: bool = True, workspace: Optional[torch.Tensor] = None,
+                       stream=None):
+    """BF16 tensor -> (FP32 image after a round trip through the 4-bit format `fmt` or None, one-element FP64 device
+    tensor holding the summed squared error): the quantization-error experiment of Section III-A."""
+    _need_cuda(src, workspace)
+    assert src.dtype == torch.bfloat16 and src.is_contiguous()
+    n = src.numel()
+    image = torch.empty(src.shape, dtype=torch.float32, device=src.device) if want_image else None
+    err = torch.empty(1, dtype=torch.float64, device=src.device)
+    need = hif4_mse_workspace(n, fmt)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=src.device)
+    _check("hif4_mse_roundtrip", lib.hif4_mse_roundtrip(src.data_ptr(), n, fmt, image.data_ptr() if want_image else None,
+                                                        err.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream(stream)))
+    return image, err
 
 
 def hif4_debug_wait_timeout(budget_ns: int, stream=None) -> None:

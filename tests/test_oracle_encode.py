@@ -546,62 +546,103 @@ def test_reencoding_decoded_units_is_stable_where_algorithm1_guarantees_it():
 
 
 # ------------------------------------------------------------------ the paper's MSE ratio
-def _round_to_grid(x, grid):
-    """Nearest value of a sorted non-negative grid, ties to the entry with even index (E2M1's even
-    mantissa), sign kept, saturating."""
-    a = np.abs(x)
-    idx = np.searchsorted(grid, a, side="left").clip(1, len(grid) - 1)
-    lo, hi = grid[idx - 1], grid[idx]
+# numpy restatements (float32 operations, one per step) of the two comparison formats of Section III-A; the oracle's
+# own C++ versions are checked against them bit for bit, against hand cases, and - together with the HiF4 encoder -
+# against the ratio the paper prints.
+_E2M1 = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6], dtype=np.float32)
+
+
+def _round_to_e2m1(a):
+    """Nearest E2M1 magnitude of non-negative float32 values, ties to the entry with even index, saturating."""
+    idx = np.searchsorted(_E2M1, a, side="left").clip(1, len(_E2M1) - 1)
+    lo, hi = _E2M1[idx - 1], _E2M1[idx]
     pick_hi = (a - lo > hi - a) | ((a - lo == hi - a) & (idx % 2 == 0))
-    return np.sign(x) * np.where(pick_hi, hi, lo)
-
-
-_E2M1 = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6], dtype=np.float64)
+    return np.where(pick_hi, hi, lo).astype(np.float32)
 
 
 def _mxfp4(x):
     """OCP MXFP4: 32-element blocks, power-of-two scale 2^(floor(log2 amax) - 2), E2M1 elements."""
-    b = x.reshape(-1, 32)
+    b = np.asarray(x, dtype=np.float32).reshape(-1, 32)
     amax = np.abs(b).max(axis=1, keepdims=True)
-    scale = np.exp2(np.floor(np.log2(np.where(amax > 0, amax, 1.0))) - 2)
-    return (_round_to_grid(b / scale, _E2M1) * scale).reshape(x.shape)
+    e = np.frexp(np.where(amax > 0, amax, 1.0))[1] - 1 - 2                 # floor(log2 amax) - 2
+    scale = np.ldexp(np.float32(1), e).astype(np.float32)
+    out = _round_to_e2m1((np.abs(b) / scale).astype(np.float32)) * scale
+    return np.copysign(np.where(amax > 0, out, 0), b).astype(np.float32).reshape(np.shape(x))
 
 
 def _e4m3(v):
-    """Round positive values to FP8-E4M3 (4-bit significand, min normal 2^-6, subnormals, max 448)."""
-    e = np.floor(np.log2(np.where(v > 0, v, 1.0))).clip(-6, None)
-    q = np.exp2(e - 3)
-    return np.minimum(np.rint(v / q) * q, 448.0)
+    """Round non-negative float32 values to FP8-E4M3 (4-bit significand, min normal 2^-6, subnormals, max 448)."""
+    v = np.asarray(v, dtype=np.float32)
+    e = (np.frexp(np.where(v > 0, v, 1.0))[1] - 1).clip(-6, None)
+    q = np.ldexp(np.float32(1), e - 3).astype(np.float32)
+    return np.minimum(np.rint(v / q) * q, np.float32(448)).astype(np.float32)
 
 
-def _nvfp4(x, pts):
-    """NVFP4: 16-element blocks, E4M3 scale = amax/6, E2M1 elements; optional per-tensor scaling of
-    the tensor's peak to 2688 = 448 * 6 beforehand."""
-    g = 2688.0 / np.abs(x).max() if pts else 1.0
-    b = (x * g).reshape(-1, 16)
+def _nvfp4(x, gain):
+    """NVFP4: 16-element blocks, E4M3 scale = amax / 6, E2M1 elements, on gain * x, divided by the gain afterwards."""
+    gain = np.float32(gain)
+    b = (np.asarray(x, dtype=np.float32) * gain).astype(np.float32).reshape(-1, 16)
     amax = np.abs(b).max(axis=1, keepdims=True)
-    scale = _e4m3(amax / 6.0)
-    safe = np.where(scale > 0, scale, 1.0)
-    return (_round_to_grid(b / safe, _E2M1) * scale).reshape(x.shape) / g
+    scale = _e4m3((amax / np.float32(6)).astype(np.float32))
+    safe = np.where(scale > 0, scale, np.float32(1))
+    d = np.where(scale > 0, _round_to_e2m1((np.abs(b) / safe).astype(np.float32)) * scale, 0).astype(np.float32)
+    return (np.copysign(d, b) / gain).astype(np.float32).reshape(np.shape(x))
+
+
+def test_comparison_format_hand_cases():
+    """E2M1 ties go to the even code (0, 1, 2, 4); E4M3 ties to the even mantissa, subnormal step 2^-9, saturation at
+    448; MXFP4 with amax = 7.5: floor(log2 7.5) - 2 = 0 -> scale 1, 7.5 saturates to 6 and 2.5 ties to 2; NVFP4 with
+    amax = 6: scale E4M3(1) = 1; with amax = 3000: 500 saturates the scale at 448, so 3000 / 448 = 6.7 clamps to 6 -> 2688."""
+    got = [oracle.e2m1_round(v) for v in (0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 5.01, 7.9, 0.2501, 0.0)]
+    assert got == [0.0, 1.0, 1.0, 2.0, 2.0, 4.0, 4.0, 6.0, 6.0, 0.5, 0.0]
+    got = [oracle.e4m3_round(v) for v in (448, 500, 2 ** -9, 0.001, 2 ** -10, 1.0625, 1.1875, 17, 18, 0.0)]
+    assert got == [448.0, 448.0, 2 ** -9, 2 ** -9, 0.0, 1.0, 1.25, 16.0, 18.0, 0.0]
+    x = np.zeros(32, dtype=np.float32); x[0], x[1], x[2], x[3] = 7.5, -2.5, 0.25, -0.3
+    want = np.zeros(32, dtype=np.float32); want[0], want[1], want[2], want[3] = 6.0, -2.0, 0.0, -0.5
+    assert np.array_equal(oracle.mxfp4_roundtrip(x), want)
+    y = np.zeros(16, dtype=np.float32); y[0], y[1], y[2] = 6.0, -1.25, 0.76
+    want = np.zeros(16, dtype=np.float32); want[0], want[1], want[2] = 6.0, -1.0, 1.0
+    assert np.array_equal(oracle.nvfp4_roundtrip(y), want)
+    z = np.zeros(16, dtype=np.float32); z[5] = -3000.0
+    assert oracle.nvfp4_roundtrip(z)[5] == -2688.0
+    assert oracle.pts_gain(z) == float(np.float32(2688.0) / np.float32(3000.0)) and oracle.pts_gain(np.zeros(16, np.float32)) == 1.0
+    assert abs(oracle.nvfp4_roundtrip(z, oracle.pts_gain(z))[5] + 3000.0) < 1e-3       # scaled to 2688, exactly representable
+
+
+def test_comparison_formats_match_their_numpy_restatement():
+    rng = np.random.default_rng(18)
+    for xexp in (0, 9, 17):
+        x = to_bf16_bits((rng.standard_normal((64, 1024)) * 0.01 * 2.0 ** xexp).astype(np.float32))
+        xf = oracle.bf16_bits_to_f64(x).astype(np.float32)
+        assert np.array_equal(oracle.mxfp4_roundtrip(xf), _mxfp4(xf))
+        assert np.array_equal(oracle.nvfp4_roundtrip(xf), _nvfp4(xf, 1.0))
+        g = oracle.pts_gain(xf)
+        assert g == float(np.float32(2688.0) / np.abs(xf).max())
+        assert np.array_equal(oracle.nvfp4_roundtrip(xf, g), _nvfp4(xf, g))
 
 
 def test_gaussian_mse_ratio_matches_the_paper(golden_dir):
     paper = paper_constants.load(golden_dir)
     rng = np.random.default_rng(8)
-    ratios_nv, ratios_mx = [], []
+    ratios_nv, ratios_mx, direct = [], [], {}
     for xexp in (0, 4, 9, 13, 17):
         x = (rng.standard_normal((256, 1024)) * 0.01 * 2.0 ** xexp).astype(np.float32)
         bits = to_bf16_bits(x)
         xd = oracle.bf16_bits_to_f64(bits)
+        xf = xd.astype(np.float32)
         hif4 = oracle.dequantize(oracle.quantize(bits, nthreads=4), oracle.FP64, nthreads=4)
         mse_h = np.mean((hif4 - xd) ** 2)
-        ratios_nv.append(np.mean((_nvfp4(xd, True) - xd) ** 2) / mse_h)
-        ratios_mx.append(np.mean((_mxfp4(xd) - xd) ** 2) / mse_h)
+        ratios_nv.append(np.mean((oracle.nvfp4_roundtrip(xf, oracle.pts_gain(xf)).astype(np.float64) - xd) ** 2) / mse_h)
+        ratios_mx.append(np.mean((oracle.mxfp4_roundtrip(xf).astype(np.float64) - xd) ** 2) / mse_h)
+        direct[xexp] = np.mean((oracle.nvfp4_roundtrip(xf).astype(np.float64) - xd) ** 2) / mse_h
     assert abs(np.mean(ratios_nv) - float(paper["mse_ratio_nvfp4"])) < 0.04, ratios_nv
     assert abs(np.mean(ratios_mx) - float(paper["mse_ratio_mxfp4"])) < 0.04, ratios_mx
     assert max(ratios_nv) - min(ratios_nv) < 0.06 and max(ratios_mx) - min(ratios_mx) < 0.06
     # "reduces the MSE by 24 %" relative to NVFP4
     assert abs((1 - 1 / np.mean(ratios_nv)) - 0.24) < 0.03
+    # the direct cast matches the scaled pipeline in the middle of E4M3's range and degrades at both ends
+    # (Section III-A: overflow and underflow near the numeric bounds of NVFP4)
+    assert abs(direct[9] - ratios_nv[2]) < 0.05 and direct[0] > 1.6 and direct[17] > 1.6
 
 
 # ------------------------------------------------------------------ brute force lower bound
