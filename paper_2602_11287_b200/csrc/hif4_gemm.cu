@@ -83,7 +83,12 @@ extern "C" hif4_status hif4_grouped_gemm_workspace(int num_groups, int64_t total
   if (num_groups < 0 || total_rows < 0 || total_rows > kGroupedMaxRows || N < 0 || K < 0 || K % kUnitElems != 0)
     return HIF4_ERR_SHAPE;
   // the tensor-core path keeps its tile table (one 16-byte entry per 128-row tile) here
-  *bytes = (K > 0 && K % 256 == 0 && total_rows > 0 && num_groups > 0) ? grouped_tc_workspace_bytes(num_groups, total_rows) : 0;
+  *bytes = 0;
+  if (K > 0 && K % 256 == 0 && total_rows > 0 && num_groups > 0) {      // the larger of the two tensor-core kernels' tables
+    const size_t single = grouped_tc_workspace_bytes(num_groups, total_rows);
+    const size_t pairs = N > 0 ? grouped_tc2_workspace_bytes(num_groups, total_rows, N) : 0;
+    *bytes = single > pairs ? single : pairs;
+  }
   return HIF4_OK;
 }
 
@@ -107,7 +112,7 @@ extern "C" hif4_status hif4_grouped_gemm(const void* A_units, const void* B_unit
                      gemm_tc_supported(A_units, B_units, total_rows, static_cast<int64_t>(num_groups) * N, N, K);
   if (tc_ok && g_gemm_path != 2 && N < (1ll << 31) - 256 && static_cast<int64_t>(num_groups) * N < (1ll << 31) - 256) {
     // CTA pairs, swapped operands: padding of small experts costs 32 rows instead of 128
-    if (!workspace || workspace_bytes < grouped_tc2_workspace_bytes(num_groups, total_rows)) return HIF4_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes < grouped_tc2_workspace_bytes(num_groups, total_rows, N)) return HIF4_ERR_WORKSPACE;
     if (!aligned(workspace, 256)) return HIF4_ERR_ALIGN;
     return launch_grouped_gemm_tc2(A_units, B_units, C, group_offsets_dev, num_groups, total_rows, N, K, ldc,
                                    workspace, st);

@@ -40,7 +40,7 @@ hif4_status launch_grouped_gemm_tc(const void* A, const void* B, float* C, const
 
 // Grouped GEMM on CTA pairs with swapped operands (weights on the MMA M side, token tiles of 32..256
 // rows on the N side); same requirements as the tensor-core path, workspace = its tile table.
-size_t grouped_tc2_workspace_bytes(int num_groups, int64_t total_rows);
+size_t grouped_tc2_workspace_bytes(int num_groups, int64_t total_rows, int64_t N);
 // (dense problems with fewer weight tiles than CTA pairs are cut along K; their workspace holds the slices' completion words)
 size_t gemm_tc2_swapped_workspace_bytes(int64_t M, int64_t N, int64_t K);
 hif4_status launch_gemm_tc2_swapped(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K,

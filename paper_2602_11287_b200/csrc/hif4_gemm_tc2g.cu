@@ -13,6 +13,14 @@
 // Pipeline, barriers and bounded waits are those of the dense CTA-pair kernel: TMA producer warp (raw
 // units, K = 256 per stage, each CTA fetches its own rows), 16 decode warps, the MMA-issuing thread
 // on rank 0 with multicast commits, 4 epilogue warps, two accumulator stages.
+//
+// Small token tiles (T <= 64, three quarters of the tiles of a Zipf-routed layer): the time of a K chunk is the
+// serial decode of two units per decode thread whatever T is, and with T / 2 <= 32 token rows per CTA almost all
+// of the 256 "token row" threads would idle.  Such a tile is therefore multiplied with TWO weight tiles at once:
+// the token-row threads decode the 128 rows of the second weight tile instead, four extra warps decode the few
+// token rows (one unit per thread and chunk, read straight from global memory into a small operand buffer of
+// their own), the MMA thread issues both products against the same token block into two accumulators, and the
+// epilogue stores both.  The unit count of those tiles halves.
 #include "hif4_common.cuh"
 #include "hif4_gemm_internal.cuh"
 #include "hif4_tc2_common.cuh"
@@ -32,13 +40,20 @@ constexpr int kTmemCols = 512;
 
 constexpr int kDecodeWarp0 = 6;
 constexpr int kDecodeThreads = 512;
-constexpr int kThreads = kDecodeWarp0 * 32 + kDecodeThreads;   // 704
-constexpr int kSmemBytes = 1024 + kDecStages * kDecStageBytes + kRawStages * kRawStageBytes + 256 + 1024;
+constexpr int kTokWarp0 = kDecodeWarp0 + kDecodeThreads / 32;  // 22: the four token warps of the small-tile mode
+constexpr int kTokThreads = 128;                               // (unit of the chunk, token row): 4 x 32
+constexpr int kSmallT = 64;                                    // token tiles up to this many rows take two weight tiles
+constexpr int kTokBufBytes = 32 * 128;                         // decoded token rows of one K = 64 block (small mode)
+constexpr int kThreads = kDecodeWarp0 * 32 + kDecodeThreads + kTokThreads;   // 832
+constexpr int kSmemBytes = 1024 + kDecStages * kDecStageBytes + kRawStages * kRawStageBytes + kDecStages * kTokBufBytes + 256 + 1024;
 
 // tcgen05.mma kind::f16 descriptor without the N field: D = F32, A = B = BF16, K-major, M = 256.
 constexpr uint32_t kInstrDescM256 = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(256 >> 4) << 24);
 
-struct TokTile { int tok0; int tok_end; int group; int T; };     // T = rows of the tile rounded up to 32
+// One work record: token rows [tok0, tok0 + T) of a group (valid below tok_end) times weight rows [w_row0, +256) of
+// that group's matrix (columns [n0, +256) of C); tiles = 2: also the next 256 weight rows (small-tile mode).
+struct WorkRec { int tok0; int tok_end; int w_row0; int n0; int T; int tiles; };
+constexpr int kTableHeaderBytes = 32;                 // record count, then the records
 
 struct GroupedParams {
   float* C;
@@ -46,8 +61,12 @@ struct GroupedParams {
   int64_t N;            // weight rows per expert = columns of C
   int num_kc;           // K / 256
   int n_wtiles;         // ceil(N / 256)
-  int max_entries;
-  const TokTile* table;     // nullptr: one dense problem of dense_rows token rows (a single tile)
+  int max_entries;          // dense problems: 1
+  const WorkRec* table;     // nullptr: one dense problem of dense_rows token rows (a single tile)
+  const int* table_count;   // number of records (written by the table kernel)
+  const uint32_t* tok_units;    // the token operand again, for the token warps of the small-tile mode
+  int64_t tok_rows;
+  int64_t upr;              // units per row
   int dense_rows;
   // Dense problems with fewer weight tiles than CTA pairs: every tile is cut into `slices` K ranges on pairs of
   // their own.  Slice 0 stores its part of C, slice s > 0 adds to it after the same epilogue warp of slice s - 1
@@ -58,54 +77,84 @@ struct GroupedParams {
   DecodeMul mul;
 };
 
-// One thread walks the offsets: every group is cut into token tiles of 256 rows, the last one padded
-// to a multiple of 32; unused entries are marked invalid.
-__global__ void build_toktile_table_kernel(const int64_t* __restrict__ offsets, int num_groups, TokTile* table,
-                                           int max_entries) {
-  __shared__ int s_total;
-  if (threadIdx.x == 0) {
-    int n = 0;
-    for (int g = 0; g < num_groups; ++g) {
-      const int64_t lo = offsets[g], hi = offsets[g + 1];
-      for (int64_t r = lo; r < hi && n < max_entries; r += kMaxTok) {
-        const int rows = static_cast<int>(hi - r < kMaxTok ? hi - r : kMaxTok);
-        table[n].tok0 = static_cast<int>(r);
-        table[n].tok_end = static_cast<int>(hi);
-        table[n].group = g;
-        table[n].T = (rows + 31) & ~31;
-        ++n;
+// Work table from the device-side offsets: every group is cut into token tiles of 256 rows, the last one padded
+// to a multiple of 32; a tile of more than kSmallT rows gives one record per 256 weight rows, a smaller one a
+// record per PAIR of weight tiles.  Thread g counts the records of group g, a block-wide scan places them, the
+// thread writes them; groups are taken 256 at a time.
+__global__ void __launch_bounds__(256)
+build_work_table_kernel(const int64_t* __restrict__ offsets, int num_groups, int64_t N, int n_wtiles, uint8_t* table_mem,
+                        int max_records) {
+  __shared__ int warp_sums[8];
+  __shared__ int s_base;
+  WorkRec* table = reinterpret_cast<WorkRec*>(table_mem + kTableHeaderBytes);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) s_base = 0;
+  __syncthreads();
+  for (int g0 = 0; g0 < num_groups; g0 += 256) {
+    const int g = g0 + threadIdx.x;
+    int64_t lo = 0, hi = 0;
+    if (g < num_groups) { lo = offsets[g]; hi = offsets[g + 1]; }
+    const int64_t rows = hi > lo ? hi - lo : 0;
+    const int64_t full = rows / kMaxTok;
+    const int rest = static_cast<int>(rows - full * kMaxTok);
+    const int rest_units = rest == 0 ? 0 : rest <= kSmallT ? (n_wtiles + 1) / 2 : n_wtiles;
+    const int mine = static_cast<int>(full) * n_wtiles + rest_units;
+    // exclusive scan of `mine` over the block
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    int before = s_base;
+    for (int w = 0; w < warp; ++w) before += warp_sums[w];
+    int n = before + incl - mine;
+    for (int64_t r = lo; r < hi; r += kMaxTok) {
+      const int t_rows = static_cast<int>(hi - r < kMaxTok ? hi - r : kMaxTok);
+      const int step = t_rows <= kSmallT ? 2 : 1;
+      for (int wt = 0; wt < n_wtiles && n < max_records; wt += step, ++n) {
+        WorkRec rec;
+        rec.tok0 = static_cast<int>(r);
+        rec.tok_end = static_cast<int>(hi);
+        rec.n0 = wt * 256;
+        rec.w_row0 = static_cast<int>(g * N) + rec.n0;
+        rec.T = (t_rows + 31) & ~31;
+        rec.tiles = step == 2 ? (wt + 1 < n_wtiles ? 2 : 3) : 1;       // 3: small-tile mode whose second weight tile does not exist
+        table[n] = rec;
       }
     }
-    s_total = n;
+    __syncthreads();
+    if (threadIdx.x == 255) s_base = before + incl;
+    __syncthreads();
   }
-  __syncthreads();
-  for (int i = s_total + threadIdx.x; i < max_entries; i += blockDim.x) {
-    table[i].tok0 = 0; table[i].tok_end = 0; table[i].group = -1; table[i].T = 0;
-  }
+  if (threadIdx.x == 0) *reinterpret_cast<int*>(table_mem) = s_base < max_records ? s_base : max_records;
 }
 
-struct Unit { int tok0; int tok_end; int T; int w_row0; int n0; int kc0; int kc1; int wt; int slice; bool valid; };
+struct Unit { int tok0; int tok_end; int T; int w_row0; int n0; int kc0; int kc1; int wt; int slice; int tiles; };
 __device__ __forceinline__ Unit unit_of(const GroupedParams& p, int u) {
   Unit r;
   if (p.table == nullptr) {                 // dense: unit = (K slice, weight tile)
     r.slice = u / p.n_wtiles; r.wt = u - r.slice * p.n_wtiles;
     r.tok0 = 0; r.tok_end = p.dense_rows; r.T = (p.dense_rows + 31) & ~31;
-    r.valid = true;
+    r.tiles = 1;
     r.n0 = r.wt * 256;
     r.w_row0 = r.n0;
     r.kc0 = static_cast<int>(static_cast<int64_t>(r.slice) * p.num_kc / p.slices);
     r.kc1 = static_cast<int>(static_cast<int64_t>(r.slice + 1) * p.num_kc / p.slices);
     return r;
   }
-  const int e = u / p.n_wtiles;
-  r.wt = u - e * p.n_wtiles; r.slice = 0;
-  const TokTile t = p.table[e];
-  r.valid = t.group >= 0;
-  r.tok0 = t.tok0; r.tok_end = t.tok_end; r.T = t.T;
-  r.n0 = r.wt * 256;
-  r.w_row0 = static_cast<int>(t.group * p.N) + r.n0;
+  const WorkRec t = p.table[u];
+  r.wt = 0; r.slice = 0;
+  r.tok0 = t.tok0; r.tok_end = t.tok_end; r.T = t.T; r.tiles = t.tiles;
+  r.n0 = t.n0;
+  r.w_row0 = t.w_row0;
   r.kc0 = 0; r.kc1 = p.num_kc;
   return r;
+}
+__device__ __forceinline__ int total_units_of(const GroupedParams& p) {
+  return p.table == nullptr ? p.n_wtiles * p.slices : *p.table_count;
 }
 
 // Decodes the two units held in raw words W[0..8], W[9..17] into decoded stages 2h and 2h+1 (skipped for
@@ -150,7 +199,8 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t dec_base = smem_base;                                        // 1024-byte aligned stages
   const uint32_t raw_base = dec_base + kDecStages * kDecStageBytes;
-  const uint32_t bar_base = raw_base + kRawStages * kRawStageBytes;
+  const uint32_t tok_base = raw_base + kRawStages * kRawStageBytes;        // 1024-byte aligned: small-mode token blocks
+  const uint32_t bar_base = tok_base + kDecStages * kTokBufBytes;
   const uint32_t raw_full = bar_base, raw_empty = bar_base + 16, dec_full = bar_base + 32, dec_empty = bar_base + 64,
                  tmem_full = bar_base + 96, tmem_empty = bar_base + 112;
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -163,7 +213,7 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-  const int total_units = p.max_entries * p.n_wtiles * p.slices;
+  const int total_units = total_units_of(p);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kRawStages; ++s) {
@@ -171,7 +221,7 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
       mbar_init(raw_empty + 8 * s, kDecodeThreads);
     }
     for (int s = 0; s < kDecStages; ++s) {
-      mbar_init(dec_full + 8 * s, kDecodeThreads / 32);   // 8 warps of each CTA per stage (used on rank 0)
+      mbar_init(dec_full + 8 * s, kDecodeThreads / 32 + 2);   // 8 decode warps + 1 token warp of each CTA per stage (used on rank 0)
       mbar_init(dec_empty + 8 * s, 1);
     }
     for (int s = 0; s < 2; ++s) {
@@ -200,15 +250,18 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
       bool ok = true;
       for (int u = pair; u < total_units && ok; u += num_pairs) {
         const Unit un = unit_of(p, u);
-        if (!un.valid) continue;
         for (int kc = un.kc0; kc < un.kc1; ++kc, ++n) {
           const uint32_t s = n & 1u, ph = (n >> 1) & 1u;
           if (!(ok = mbar_wait(raw_empty + 8 * s, ph ^ 1u, abort_flag, 128))) break;
           mbar_expect_tx(raw_full + 8 * s, kRawStageBytes);
           const uint32_t dst = raw_base + s * kRawStageBytes;
           tma_load_2d(dst, &tmW, kc * kRawRowBytes, un.w_row0 + static_cast<int>(rank) * kWRows, raw_full + 8 * s);
-          tma_load_2d(dst + kRawHalfBytes, &tmTok, kc * kRawRowBytes, un.tok0 + static_cast<int>(rank) * (un.T >> 1),
-                      raw_full + 8 * s);
+          if (un.tiles == 1)
+            tma_load_2d(dst + kRawHalfBytes, &tmTok, kc * kRawRowBytes, un.tok0 + static_cast<int>(rank) * (un.T >> 1),
+                        raw_full + 8 * s);
+          else            // small-tile mode: the second weight tile takes the place of the token rows
+            tma_load_2d(dst + kRawHalfBytes, &tmW, kc * kRawRowBytes, un.w_row0 + 256 + static_cast<int>(rank) * kWRows,
+                        raw_full + 8 * s);
         }
       }
     }
@@ -219,7 +272,6 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
       bool ok = true;
       for (int u = pair; u < total_units && ok; u += num_pairs) {
         const Unit un = unit_of(p, u);
-        if (!un.valid) continue;
         const uint32_t acc = ucount & 1u, aph = (ucount >> 1) & 1u;
         if (!(ok = mbar_wait_cluster(tmem_empty + 8 * acc, aph ^ 1u, abort_flag))) break;
         tc_fence_after();
@@ -233,10 +285,24 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
             if (!(ok = mbar_wait_cluster(dec_full + 8 * st, n & 1u, abort_flag))) break;
             tc_fence_after();
             const uint64_t adesc = make_desc(dec_base + st * kDecStageBytes);                  // weights: M side
-            const uint64_t bdesc = make_desc(dec_base + st * kDecStageBytes + kDecHalfBytes);  // tokens: N side
+            if (un.tiles == 1) {
+              const uint64_t bdesc = make_desc(dec_base + st * kDecStageBytes + kDecHalfBytes);  // tokens: N side
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              tc2_mma(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, ((kc - un.kc0) | i | kk) != 0 ? 1u : 0u);
+              for (int kk = 0; kk < 4; ++kk)
+                tc2_mma(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, ((kc - un.kc0) | i | kk) != 0 ? 1u : 0u);
+            } else {
+              // small-tile mode: both halves of the stage are weight tiles, the tokens sit in their own block
+              const uint64_t a2desc = make_desc(dec_base + st * kDecStageBytes + kDecHalfBytes);
+              const uint64_t bdesc = make_desc(tok_base + st * kTokBufBytes);
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk)
+                tc2_mma(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, ((kc - un.kc0) | i | kk) != 0 ? 1u : 0u);
+              if (un.tiles == 2) {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                  tc2_mma(d_tmem + 128, a2desc + 2 * kk, bdesc + 2 * kk, idesc, ((kc - un.kc0) | i | kk) != 0 ? 1u : 0u);
+              }
+            }
             tc2_commit_both(dec_empty + 8 * st);
           }
         }
@@ -252,36 +318,39 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
     uint32_t ucount = 0;
     for (int u = pair; u < total_units; u += num_pairs) {
       const Unit un = unit_of(p, u);
-      if (!un.valid) continue;
       const uint32_t acc = ucount & 1u, aph = (ucount >> 1) & 1u;
       if (!__all_sync(0xFFFFFFFFu, mbar_wait(tmem_full + 8 * acc, aph, abort_flag, 256))) break;
       tc_fence_after();
-      const int64_t col = static_cast<int64_t>(un.n0) + rank * kWRows + q * 32 + lane;      // column of C = weight row
-      const bool col_ok = col < p.N;
       const int chunks = un.T >> 4;
       // K-sliced dense tile: slices after the first add to what the previous slice has left in C
       const bool adds = un.slice > 0;
       unsigned int* my_flag = p.slices > 1 ? p.flags + (static_cast<size_t>(un.wt) * p.slices + un.slice) * 8 + rank * 4 + q : nullptr;
       if (adds && !__all_sync(0xFFFFFFFFu, wait_word(my_flag - 8, 1u, abort_flag))) break;
+      const int n_acc = un.tiles == 2 ? 2 : 1;   // small-tile mode: a second accumulator 128 columns further, 256 columns of C further
 #pragma unroll 1
-      for (int c = 0; c < chunks; ++c) {
-        uint32_t r[16];
-        tc_ld16(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kMaxTok + c * 16, r);
-        tc_wait_ld();
-        if (c == chunks - 1) {                   // accumulator fully read: hand it back before the stores
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + 8 * acc);
-        }
-        const int tok = un.tok0 + c * 16;
-        float* cp = p.C + static_cast<int64_t>(tok) * p.ldc + col;
-#pragma unroll
-        for (int v = 0; v < 16; ++v)
-          if (col_ok && tok + v < un.tok_end) {
-            float* dst = cp + static_cast<int64_t>(v) * p.ldc;
-            if (adds) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst), "f"(__uint_as_float(r[v])) : "memory");
-            else *dst = __uint_as_float(r[v]);
+      for (int a = 0; a < n_acc; ++a) {
+        const int64_t col = static_cast<int64_t>(un.n0) + a * 256 + rank * kWRows + q * 32 + lane;   // column of C = weight row
+        const bool col_ok = col < p.N;
+#pragma unroll 1
+        for (int c = 0; c < chunks; ++c) {
+          uint32_t r[16];
+          tc_ld16(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kMaxTok + a * 128 + c * 16, r);
+          tc_wait_ld();
+          if (a == n_acc - 1 && c == chunks - 1) {   // accumulator fully read: hand it back before the stores
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + 8 * acc);
           }
+          const int tok = un.tok0 + c * 16;
+          float* cp = p.C + static_cast<int64_t>(tok) * p.ldc + col;
+#pragma unroll
+          for (int v = 0; v < 16; ++v)
+            if (col_ok && tok + v < un.tok_end) {
+              float* dst = cp + static_cast<int64_t>(v) * p.ldc;
+              if (adds) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst), "f"(__uint_as_float(r[v])) : "memory");
+              else *dst = __uint_as_float(r[v]);
+            }
+        }
       }
       if (p.slices > 1 && un.slice + 1 < p.slices) {      // the next slice may add to these columns now
         __threadfence();
@@ -289,6 +358,46 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
         if (lane == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(my_flag), "r"(1u) : "memory");
       }
       ++ucount;
+    }
+  } else if (warp >= kTokWarp0) {
+    // ---------------------------------------------------------------- token warps (small-tile mode): warp w = unit w of the chunk
+    const int w = warp - kTokWarp0;
+    const uint32_t r7 = static_cast<uint32_t>(lane) & 7u;
+    const uint32_t dec_row = tok_base + static_cast<uint32_t>(w) * kTokBufBytes + static_cast<uint32_t>(lane) * 128u;
+    uint32_t chunk_addr[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) chunk_addr[j] = dec_row + ((static_cast<uint32_t>(j) ^ r7) << 4);
+    const uint32_t my_empty = dec_empty + 8 * w;
+    const uint32_t my_full_leader = mapa(dec_full, 0) + 8 * w;
+    uint32_t n = 0;
+    bool ok = true;
+    for (int u = pair; u < total_units && ok; u += num_pairs) {
+      const Unit un = unit_of(p, u);
+      const int64_t tok = static_cast<int64_t>(un.tok0) + rank * (un.T >> 1) + lane;      // this lane's token row
+      const bool active = un.tiles != 1 && lane < (un.T >> 1) && tok < p.tok_rows;
+      const uint32_t* src = p.tok_units + (tok * p.upr + static_cast<int64_t>(un.kc0) * kRawUnits + w) * kUnitWords;
+      uint32_t W[9];
+      if (active) {
+#pragma unroll
+        for (int i = 0; i < 9; ++i) W[i] = __ldg(src + i);
+      }
+      for (int kc = un.kc0; kc < un.kc1 && ok; ++kc, ++n) {
+        uint32_t Wn[9];
+        const bool more = active && kc + 1 < un.kc1;          // the next chunk's unit is requested before this one is decoded
+        if (more) {
+#pragma unroll
+          for (int i = 0; i < 9; ++i) Wn[i] = __ldg(src + (kc + 1 - un.kc0) * (kRawUnits * kUnitWords) + i);
+        }
+        if (!(ok = __all_sync(0xFFFFFFFFu, mbar_wait(my_empty, (n & 1u) ^ 1u, abort_flag, 32)))) break;
+        if (active) decode_unit_balanced(W[0], &W[1], chunk_addr, 0u, lut, p.mul);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(my_full_leader);
+        if (more) {
+#pragma unroll
+          for (int i = 0; i < 9; ++i) W[i] = Wn[i];
+        }
+      }
     }
   } else {
     // ---------------------------------------------------------------- decode
@@ -307,8 +416,7 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
     bool ok = true;
     for (int u = pair; u < total_units && ok; u += num_pairs) {
       const Unit un = unit_of(p, u);
-      if (!un.valid) continue;
-      const bool active = row < 128 || (row - 128) < (un.T >> 1);
+      const bool active = row < 128 || un.tiles != 1 || (row - 128) < (un.T >> 1);    // small-tile mode: rows 128.. are weight rows too
       for (int kc = un.kc0; kc < un.kc1 && ok; ++kc, ++n) {
         const uint32_t s = n & 1u, ph = (n >> 1) & 1u;
         if (!(ok = __all_sync(0xFFFFFFFFu, mbar_wait(raw_full + 8 * s, ph, abort_flag)))) break;
@@ -353,6 +461,7 @@ hif4_status launch_swapped(const void* A, const void* B, int64_t a_rows, int64_t
   const int64_t upr = K / kUnitElems;
   if (!make_unit_map(&tmTok, A, a_rows, upr, 128) || !make_unit_map(&tmW, B, b_rows, upr, kWRows)) return HIF4_ERR_CUDA;
   p.num_kc = static_cast<int>(K / (kRawUnits * kUnitElems));
+  p.upr = upr;
   p.n_wtiles = static_cast<int>(ceil_div64(p.N, 256));
   p.error_word = device_error_word();
   if (!p.error_word) return HIF4_ERR_CUDA;
@@ -407,23 +516,28 @@ hif4_status launch_gemm_tc2_swapped(const void* A, const void* B, float* C, int6
   return launch_swapped(A, B, M, N, p, K, st);
 }
 
-size_t grouped_tc2_workspace_bytes(int num_groups, int64_t total_rows) {
-  const int64_t max_entries = ceil_div64(total_rows, kMaxTok) + num_groups;
-  return static_cast<size_t>((max_entries * static_cast<int64_t>(sizeof(TokTile)) + 255) / 256 * 256);
+size_t grouped_tc2_workspace_bytes(int num_groups, int64_t total_rows, int64_t N) {
+  const int64_t max_records = (ceil_div64(total_rows, kMaxTok) + num_groups) * ceil_div64(N, 256);
+  return static_cast<size_t>((kTableHeaderBytes + max_records * static_cast<int64_t>(sizeof(WorkRec)) + 255) / 256 * 256);
 }
 
 hif4_status launch_grouped_gemm_tc2(const void* A, const void* B, float* C, const int64_t* offsets, int num_groups,
                                     int64_t total_rows, int64_t N, int64_t K, int64_t ldc, void* workspace,
                                     cudaStream_t st) {
-  const int max_entries = static_cast<int>(ceil_div64(total_rows, kMaxTok) + num_groups);
-  TokTile* table = static_cast<TokTile*>(workspace);
-  build_toktile_table_kernel<<<1, 256, 0, st>>>(offsets, num_groups, table, max_entries);
+  const int n_wtiles = static_cast<int>(ceil_div64(N, 256));
+  const int64_t max_records = (ceil_div64(total_rows, kMaxTok) + num_groups) * n_wtiles;
+  if (max_records > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
+  uint8_t* table_mem = static_cast<uint8_t*>(workspace);
+  build_work_table_kernel<<<1, 256, 0, st>>>(offsets, num_groups, N, n_wtiles, table_mem, static_cast<int>(max_records));
   note_launch();
   if (cudaGetLastError() != cudaSuccess) return HIF4_ERR_CUDA;
   GroupedParams p{};
   p.C = C; p.ldc = ldc; p.N = N;
-  p.max_entries = max_entries;
-  p.table = table;
+  p.max_entries = static_cast<int>(max_records / n_wtiles);
+  p.table = reinterpret_cast<const WorkRec*>(table_mem + kTableHeaderBytes);
+  p.table_count = reinterpret_cast<const int*>(table_mem);
+  p.tok_units = static_cast<const uint32_t*>(A);
+  p.tok_rows = total_rows;
   return launch_swapped(A, B, total_rows, static_cast<int64_t>(num_groups) * N, p, K, st);
 }
 
