@@ -7,9 +7,11 @@ using namespace hif4;
 namespace {
 // Test hook (hif4_debug_set_gemm_path): 0 = choose by shape, 1 = CUDA-core kernel only, 2 = single-CTA
 // tensor-core kernel whenever it is legal, 3 = CTA-pair tensor-core kernel whenever it is legal,
-// 4 = weight-streaming kernel whenever it is legal (M <= kGemvMaxM).
+// 4 = weight-streaming kernel whenever it is legal (M <= kGemvMaxM), 6 = hif4_linear converts BF16 activations inside
+// the CTA-pair kernel whenever that is legal (hif4_gemm itself behaves as under 0).
 int g_gemm_path = 0;
 constexpr int64_t kPairMinM = 129;      // below that a 256-row pair tile would be half empty
+constexpr int64_t kFuseMaxColumnTiles = 0;   // hif4_linear: in-kernel conversion for C with at most this many 256-column tiles
 constexpr int64_t kGroupedMaxRows = (1ll << 31) - 257;   // tile tables keep row numbers (and row + tile height) in 32-bit ints
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -41,7 +43,7 @@ extern "C" hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size
 }
 
 extern "C" hif4_status hif4_debug_set_gemm_path(int path) {
-  if (path < 0 || path > 4) return HIF4_ERR_DTYPE;
+  if (path < 0 || path > 6) return HIF4_ERR_DTYPE;
   g_gemm_path = path;
   return HIF4_OK;
 }
@@ -160,6 +162,20 @@ extern "C" hif4_status hif4_linear(const void* X, hif4_dtype dt, int64_t ld_x, c
       gemv_linear_supported(X, dt, ld_x, W_units, M, N, K))
     return launch_gemv_linear(X, dt, ld_x, mode == HIF4_RHA, W_units, Y, M, N, K, ldy, x_units + x_bytes,
                               static_cast<cudaStream_t>(stream));
+  // Many rows: the conversion can also run inside the pair kernel's A-side decode threads (once per column tile of
+  // C).  Measured against the two launches it loses on every shape, even with a single column tile (M = 4096,
+  // K = 4096: N = 256 62 vs 44 us, N = 1024 100 vs 52 us, N = 14336 1149 vs 381 us): Algorithm 1 costs about 2.6 times
+  // the decode per element and sits on the critical path of every K chunk.  kFuseMaxColumnTiles = 0 therefore keeps
+  // the default on two launches; the test hook (path 6) still reaches the fused kernel, whose result is bit-identical.
+  if (dt == HIF4_BF16 && mode == HIF4_RNE && K > 0 && M >= kPairMinM && X && W_units && Y && ldy >= N &&
+      (g_gemm_path == 6 || (g_gemm_path == 0 && ceil_div64(N, 256) <= kFuseMaxColumnTiles)) && aligned(X, 16) &&
+      ld_x >= K && (ld_x * 2) % 16 == 0 && aligned(W_units, 4) && aligned(Y, 4) &&
+      gemm_tc2_supported(W_units, W_units, M, N, K)) {
+    size_t pair_bytes = gemm_tc2_workspace_bytes(M, N, K);
+    if (pair_bytes > workspace_bytes - x_bytes) return HIF4_ERR_WORKSPACE;
+    return launch_gemm_tc2_fused_bf16(X, ld_x, W_units, Y, M, N, K, ldy, x_units + x_bytes, workspace_bytes - x_bytes,
+                                      static_cast<cudaStream_t>(stream));
+  }
   if (K > 0) {
     const hif4_status q = hif4_quantize(X, dt, M, K, ld_x, x_units, mode, stream);
     if (q != HIF4_OK) return q;

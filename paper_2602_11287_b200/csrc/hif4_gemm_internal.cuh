@@ -21,6 +21,10 @@ bool gemm_tc2_supported(const void* A, const void* B, int64_t M, int64_t N, int6
 size_t gemm_tc2_workspace_bytes(int64_t M, int64_t N, int64_t K);
 hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,
                             void* workspace, size_t workspace_bytes, cudaStream_t st);
+// The same kernel with the activation conversion inside: X is [M, K] BF16 (row stride ld_x elements, rows 16-byte
+// aligned), converted with Algorithm 1 (round-half-to-even) by the A-side decode threads, once per column tile.
+hif4_status launch_gemm_tc2_fused_bf16(const void* X, int64_t ld_x, const void* B, float* C, int64_t M, int64_t N, int64_t K,
+                                       int64_t ldc, void* workspace, size_t workspace_bytes, cudaStream_t st);
 // Weight-streaming path for M <= kGemvMaxM tokens (mma.sync on register-decoded weights): needs
 // K % 256 == 0, 16-byte aligned B and a workspace of gemv_workspace_bytes (the decoded tokens).
 constexpr int64_t kGemvMaxM = 32;

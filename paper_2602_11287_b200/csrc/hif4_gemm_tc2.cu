@@ -26,6 +26,7 @@
 // the kernel returns.
 #include "hif4_common.cuh"
 #include "hif4_gemm_internal.cuh"
+#include "hif4_quantize_device.cuh"
 #include "hif4_tc_common.cuh"
 #include "hif4_tc2_common.cuh"
 
@@ -84,6 +85,10 @@ struct Gemm2Params {
   int sk_tile0;
   unsigned int* flags;      // [tail_tiles or pairs + 1][slices][8]: "this epilogue warp's rows of this slice are in C" (zero at launch)
   DecodeMul mul;
+  // Fused activation conversion (kFusedA): the A operand is not packed units but BF16 activations [M, K], row stride
+  // ld_x elements; the A-side decode threads run Algorithm 1 on the two units they are about to decode.
+  const uint16_t* x;
+  int64_t ld_x;
 };
 
 constexpr int kMaxSlices = 4;
@@ -181,6 +186,7 @@ __device__ __forceinline__ bool decode_two_units(const uint32_t (&W)[18], const 
   return true;
 }
 
+template <bool kFusedA>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                 const __grid_constant__ CUtensorMap tmC, const Gemm2Params p) {
@@ -243,9 +249,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         for (int kc = w.kc0; kc < w.kc1; ++kc, ++n) {
           const uint32_t s = n & 1u, ph = (n >> 1) & 1u;
           if (!(ok = mbar_wait(raw_empty + 8 * s, ph ^ 1u, abort_flag, 128))) break;
-          mbar_expect_tx(raw_full + 8 * s, kRawStageBytes);
+          mbar_expect_tx(raw_full + 8 * s, kFusedA ? kRawHalfBytes : kRawStageBytes);
           const uint32_t dst = raw_base + s * kRawStageBytes;
-          tma_load_2d(dst, &tmA, kc * kRawRowBytes, w.m0 + static_cast<int>(rank) * kRows, raw_full + 8 * s);
+          if (!kFusedA) tma_load_2d(dst, &tmA, kc * kRawRowBytes, w.m0 + static_cast<int>(rank) * kRows, raw_full + 8 * s);
           tma_load_2d(dst + kRawHalfBytes, &tmB, kc * kRawRowBytes, w.n0 + static_cast<int>(rank) * kRows,
                       raw_full + 8 * s);
         }
@@ -396,6 +402,34 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const WorkItem w = work_item(p, pair, num_pairs, i);
       for (int kc = w.kc0; kc < w.kc1 && ok; ++kc, ++n) {
         const uint32_t s = n & 1u, ph = (n >> 1) & 1u;
+        if (kFusedA && row < kRows) {
+          // A rows: 128 BF16 activations of this row (units 2h, 2h+1 of the chunk) from global memory, converted with
+          // Algorithm 1 (round-half-to-even) by this thread, then decoded like packed units.  Rows past M read as zeros.
+          const int64_t gr = static_cast<int64_t>(w.m0) + rank * kRows + row;
+          uint32_t W[18];
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            uint4 v[8];
+            if (gr < p.M) {
+              const uint4* src = reinterpret_cast<const uint4*>(p.x + gr * p.ld_x + static_cast<int64_t>(kc) * 256 + (2 * h + u) * 64);
+#pragma unroll
+              for (int g = 0; g < 8; ++g) v[g] = __ldg(src + g);
+            } else {
+#pragma unroll
+              for (int g = 0; g < 8; ++g) v[g] = make_uint4(0u, 0u, 0u, 0u);
+            }
+            uint32_t codes[8], meta;
+            encode_unit_bf16_single<false>(v, codes, meta);
+            W[9 * u] = meta;
+#pragma unroll
+            for (int g = 0; g < 8; ++g) W[9 * u + 1 + g] = codes[g];
+          }
+          // the raw stage holds only B rows here, but its barriers are shared by all decode threads
+          if (!(ok = __all_sync(0xFFFFFFFFu, mbar_wait(raw_full + 8 * s, ph, abort_flag)))) break;
+          mbar_arrive(raw_empty + 8 * s);
+          ok = decode_two_units(W, chunk_addr, lut, p.mul, dec_empty0, dec_full0_leader, (n & 1u) ^ 1u, abort_flag);
+          continue;
+        }
         if (!(ok = __all_sync(0xFFFFFFFFu, mbar_wait(raw_full + 8 * s, ph, abort_flag)))) break;
         uint32_t L[20];
         const uint32_t src = raw_base + s * kRawStageBytes + raw_row;
@@ -508,14 +542,21 @@ bool gemm_tc2_supported(const void* A, const void* B, int64_t M, int64_t N, int6
   return M < (1ll << 31) - kPairM && N < (1ll << 31) - kPairN && sm_count() >= 2;
 }
 
-hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,
-                            void* workspace, size_t workspace_bytes, cudaStream_t st) {
-  static uint64_t smem_opt_in = 0;
-  if (!ensure_dynamic_smem(gemm_tc2_kernel, kSmemBytes, smem_opt_in)) return HIF4_ERR_CUDA;
+// x != nullptr: the A operand is BF16 activations converted inside the kernel (A is then unused).
+static hif4_status launch_gemm_tc2_any(const void* A, const uint16_t* x, int64_t ld_x, const void* B, float* C, int64_t M,
+                                       int64_t N, int64_t K, int64_t ldc, void* workspace, size_t workspace_bytes,
+                                       cudaStream_t st) {
+  static uint64_t smem_opt_in = 0, smem_opt_in_fused = 0;
+  if (!(x ? ensure_dynamic_smem(gemm_tc2_kernel<true>, kSmemBytes, smem_opt_in_fused)
+          : ensure_dynamic_smem(gemm_tc2_kernel<false>, kSmemBytes, smem_opt_in)))
+    return HIF4_ERR_CUDA;
   CUtensorMap tmA, tmB;
   const int64_t upr = K / kUnitElems;
-  if (!make_unit_map(&tmA, A, M, upr, kRows) || !make_unit_map(&tmB, B, N, upr, kRows)) return HIF4_ERR_CUDA;
+  if (!make_unit_map(&tmB, B, N, upr, kRows)) return HIF4_ERR_CUDA;
+  if (x) tmA = tmB;                                   // placeholder: the fused kernel never loads A through TMA
+  else if (!make_unit_map(&tmA, A, M, upr, kRows)) return HIF4_ERR_CUDA;
   Gemm2Params p{};
+  p.x = x; p.ld_x = ld_x;
   p.C = C; p.ldc = ldc; p.M = M; p.N = N;
   p.num_kc = static_cast<int>(K / (kRawUnits * kUnitElems));
   p.n_tiles = static_cast<int>(ceil_div64(N, kPairN));
@@ -544,9 +585,20 @@ hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, i
     if (cudaMemsetAsync(p.flags, 0, pl.flag_bytes, st) != cudaSuccess) return HIF4_ERR_CUDA;
   }
   const int pairs = p.full_rounds == 0 && p.sk_tiles == 0 ? p.tail_tiles * p.slices : pl.pairs;      // a single round: one pair per slice
-  gemm_tc2_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tmA, tmB, tmC, p);
+  if (x) gemm_tc2_kernel<true><<<2 * pairs, kThreads, kSmemBytes, st>>>(tmA, tmB, tmC, p);
+  else gemm_tc2_kernel<false><<<2 * pairs, kThreads, kSmemBytes, st>>>(tmA, tmB, tmC, p);
   note_launch();
   return launch_status();
+}
+
+hif4_status launch_gemm_tc2(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,
+                            void* workspace, size_t workspace_bytes, cudaStream_t st) {
+  return launch_gemm_tc2_any(A, nullptr, 0, B, C, M, N, K, ldc, workspace, workspace_bytes, st);
+}
+
+hif4_status launch_gemm_tc2_fused_bf16(const void* X, int64_t ld_x, const void* B, float* C, int64_t M, int64_t N, int64_t K,
+                                       int64_t ldc, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+  return launch_gemm_tc2_any(nullptr, static_cast<const uint16_t*>(X), ld_x, B, C, M, N, K, ldc, workspace, workspace_bytes, st);
 }
 
 }  // namespace hif4

@@ -116,6 +116,37 @@ __device__ __forceinline__ void encode_unit_bf16_pair(const uint4 (&v)[4], int l
   meta_out = meta;
 }
 
+// The same unit held by ONE thread: v[g] is level-2 group g (8 elements, 16 bytes).  Same steps, same helpers, so the
+// same bits as the two-lane form; used where a GEMM's operand-decode thread converts the activations it is about to
+// decode (one unit per thread and step), with no partner lane to share the work with.
+template <bool kRHA>
+__device__ __forceinline__ void encode_unit_bf16_single(const uint4 (&v)[8], uint32_t (&codes)[8], uint32_t& meta_out) {
+  constexpr uint32_t kAbs = 0x7FFF7FFFu;
+  uint32_t vm = 0u;
+#pragma unroll
+  for (int g = 0; g < 8; ++g)
+    vm = umax2(vm, umax2(umax2(v[g].x & kAbs, v[g].y & kAbs), umax2(v[g].z & kAbs, v[g].w & kAbs)));
+  vm = hmax_halves(vm);
+  const bool unit_nan = vm > 0x7F80u;
+  const uint32_t sf = mul_bf16x2(vm, 0x3E12u) & 0xFFFFu;             // Vmax * (1/7)_BF16
+  const uint32_t byte = e6m2_from_bits<7, kRHA>(sf);
+  const uint32_t lut = prmt(0x122B4D80u, 0u, (byte & 3u) | 0x4440u);
+  const uint32_t rec2 = (lut + 0x5700u - ((byte & 0xFCu) << 5)) * 0x10001u;
+  uint32_t meta = byte;
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
+    uint32_t e8, e16a, e16b;
+    codes[g] = encode_group_bf16<kRHA>(v[g].x, v[g].y, v[g].z, v[g].w, rec2, e8, e16a, e16b);
+    meta |= (e8 << (8 + g)) | ((e16a + 2u * e16b) << (16 + 2 * g));
+  }
+  if (unit_nan) {                                      // NaN unit: E6M2 = NaN, all else zero
+    meta = 0xFFu;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) codes[g] = 0u;
+  }
+  meta_out = meta;
+}
+
 // ----------------------------------------------------------------------------- FP32 form (FP32 and FP16 sources)
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   uint4 v;

@@ -493,6 +493,38 @@ def test_linear_with_few_rows_quantizes_inside_the_token_preparation(hif4, M, N,
     assert hif4.hif4_last_device_status() == 0
 
 
+@pytest.mark.parametrize("M,N,K", [(129, 300, 256), (300, 520, 1024), (1000, 257, 768), (513, 1024, 2048), (4096, 1024, 512)])
+def test_linear_with_many_rows_can_convert_inside_the_pair_kernel(hif4, M, N, K):
+    """M > 128 rows of BF16 activations, conversion forced into the CTA-pair kernel (the A-side decode threads run
+    Algorithm 1 on the units they decode, once per column tile): one launch (plus the flag memset where tiles are
+    split along K), and exactly the bits of hif4_quantize followed by hif4_gemm -- on a strided source with spikes,
+    NaN and Inf rows and a ragged last row tile."""
+    g = torch.Generator(device="cuda"); g.manual_seed(M + 7 * N + K)
+    wide = torch.randn(M, K + 64, generator=g, device="cuda").to(torch.bfloat16)
+    x = wide[:, 64:]                                      # row stride K + 64
+    x[0, 5] = 1000.0
+    x[M // 2, 70] = float("nan")
+    x[M - 1, 129] = float("-inf")
+    w = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
+    want = hif4.hif4_gemm(hif4.hif4_quantize(x), w)
+    hif4.hif4_debug_set_gemm_path(6)
+    try:
+        before = hif4.launch_count()
+        y = hif4.hif4_linear(x, w)
+        assert hif4.launch_count() - before == 1, "conversion and GEMM in one kernel"
+        y_rha = hif4.hif4_linear(x, w, mode=1)            # half-away rounding is not fused: two launches, same contract
+    finally:
+        hif4.hif4_debug_set_gemm_path(0)
+    assert torch.equal(y.view(torch.int32), want.view(torch.int32)), "in-kernel conversion differs from quantize + GEMM"
+    assert torch.equal(y_rha.view(torch.int32), hif4.hif4_gemm(hif4.hif4_quantize(x, 1), w).view(torch.int32))
+    xq = oracle.quantize(wl.bf16_to_u16_numpy(x.contiguous()), nthreads=8)
+    ref, refabs = oracle.gemm_f64(xq, w.cpu().numpy(), nthreads=8)
+    got = y.cpu().numpy().astype(np.float64)
+    nan = np.isnan(ref)
+    assert np.array_equal(np.isnan(got), nan) and np.all(np.abs(got - ref)[~nan] <= TOL * refabs[~nan] + 1e-300)
+    assert hif4.hif4_last_device_status() == 0
+
+
 # ------------------------------------------------------------------ failure reporting
 def test_a_bounded_wait_that_runs_out_is_reported_once_and_the_context_stays_usable(hif4):
     """A kernel waits, with the library's bounded-wait helper and a 1 ms budget, on an mbarrier that nobody arrives
