@@ -304,7 +304,7 @@ def run_cuda(args):
 
     # The same step repeated for at least SUSTAINED_SECONDS: long enough for the clocks to settle under the power
     # limit and for the sampler to see it (the K timed steps above may last only milliseconds).
-    sus_steps = max(args.steps, int(SUSTAINED_SECONDS * 1e3 / max(ms_per_step, 1e-3)) + 1)
+    sus_steps = args.steps if args.no_sustained else max(args.steps, int(SUSTAINED_SECONDS * 1e3 / max(ms_per_step, 1e-3)) + 1)
     sus_events = []
     s_start, s_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -853,6 +853,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="do not stretch the second timed region to 1.5 s (for launch lists under ncu)")
     ap.add_argument("--no-per-config", action="store_true", help="skip the per_config block (configurations 1, 3, 4, 5)")
     ap.add_argument("--no-graph", action="store_true", help="launch the decode-shaped linears directly instead of replaying a CUDA graph")
     ap.add_argument("--gemm-path", type=int, default=0, help="with --case: kernel selection, see hif4_debug_set_gemm_path")
