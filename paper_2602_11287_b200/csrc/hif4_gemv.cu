@@ -14,6 +14,10 @@
 //      decodes word after word straight into the A fragments (k slots 2q, 2q+1, 2q+8, 2q+9 of every MMA
 //      come from unit q on both operands, so the K order is permuted the same way on both sides).
 //      The K slices of a pair are summed through shared memory in a fixed order.
+//   3. Up to eight tokens and K <= 6144 (kSrc 1, 2): no token kernel at all.  Every CTA decodes the few tokens itself
+//      (from packed units, or from BF16 activations that it first converts with Algorithm 1) into a resident block of
+//      shared memory before its main loop, while its producer warp is already streaming weights; one launch per
+//      product instead of two, which is most of the time of the small shapes.
 // Results are deterministic (no atomics).  Every mbarrier wait is bounded.
 #include "hif4_common.cuh"
 #include "hif4_gemm_internal.cuh"
@@ -34,8 +38,14 @@ constexpr int kMaxStages = 16;
 constexpr int kGemvWarpsMany = 31, kGemvWarpsFew = 24;
 constexpr int kRingBudget = 176 * 1024;              // bytes of shared memory given to the ring of stages
 
+constexpr int kSrcWorkspace = 0, kSrcUnits = 1, kSrcBf16 = 2;   // where the streaming kernel gets its tokens from
+constexpr int kResidentMaxBytes = 96 * 1024;          // resident tokens: K / 256 chunks of 4 KB (one n-tile)
+
 struct GemvParams {
   const uint32_t* A;        // [M, K/64] units (tokens)
+  const uint16_t* X;        // kSrcBf16: [M, K] BF16 activations, row stride ld_x elements
+  int64_t ld_x;
+  int rha;                  // kSrcBf16: rounding mode of the conversion
   uint8_t* tokens;          // workspace: [K/256][tiles][8 words][8 tokens][4 units][16 B]
   float* C;
   int64_t ldc;
@@ -203,6 +213,66 @@ gemv_quantize_tokens32_kernel(const Src* __restrict__ X, int64_t ld_x, int M, in
   }
 }
 
+// Resident tokens (one n-tile of eight tokens, all K): the consumer warps of a CTA build them before the main loop.
+// From packed units: task (token n, unit U).
+__device__ __forceinline__ void build_tokens_from_units(const uint32_t* __restrict__ A, int M, int64_t upr, uint8_t* tok,
+                                                        int tid, int nthreads) {
+  for (int64_t idx = tid; idx < 8 * upr; idx += nthreads) {
+    const int n = static_cast<int>(idx / upr);
+    const int64_t U = idx - static_cast<int64_t>(n) * upr;
+    uint8_t* dst = tok + ((U >> 2) * 8) * kTokChunkBytes + ((n & 7) * 4 + (U & 3)) * 16;
+    if (n >= M) {
+#pragma unroll
+      for (int W = 0; W < 8; ++W) *reinterpret_cast<uint4*>(dst + W * kTokChunkBytes) = make_uint4(0u, 0u, 0u, 0u);
+      continue;
+    }
+    const uint32_t* unit = A + (static_cast<int64_t>(n) * upr + U) * kUnitWords;
+    const uint32_t meta = __ldg(unit);
+#pragma unroll
+    for (int W = 0; W < 8; W += 2) {
+      uint32_t r[8];
+      decode_two_words(meta, W, __ldg(unit + 1 + W), __ldg(unit + 2 + W), r);
+      *reinterpret_cast<uint4*>(dst + W * kTokChunkBytes) = make_uint4(r[0], r[1], r[2], r[3]);
+      *reinterpret_cast<uint4*>(dst + (W + 1) * kTokChunkBytes) = make_uint4(r[4], r[5], r[6], r[7]);
+    }
+  }
+}
+// From BF16 activations: Algorithm 1 with two lanes per unit (the streaming quantizer's own code), then Eq. 2 of the
+// unit just encoded.  Whole warps take part: 16 * upr lane tasks, a multiple of 32.
+template <bool kRHA>
+__device__ __forceinline__ void build_tokens_from_bf16(const uint16_t* __restrict__ X, int64_t ld_x, int M, int64_t upr,
+                                                       uint8_t* tok, int tid, int nthreads) {
+  for (int64_t idx = tid; idx < 16 * upr; idx += nthreads) {      // nthreads is a multiple of 32: warps stay whole
+    const int l = static_cast<int>(idx & 1);
+    const int64_t pair = idx >> 1;
+    const int n = static_cast<int>(pair / upr);
+    const int64_t U = pair - static_cast<int64_t>(n) * upr;
+    uint4 v[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) v[c] = make_uint4(0u, 0u, 0u, 0u);
+    if (n < M) {
+      const uint4* src = reinterpret_cast<const uint4*>(X + static_cast<int64_t>(n) * ld_x + U * kUnitElems) + l;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) v[c] = __ldg(src + 2 * c);
+    }
+    uint32_t codes[4], meta;
+    encode_unit_bf16_pair<kRHA>(v, l, codes, meta);
+    uint8_t* dst = tok + ((U >> 2) * 8) * kTokChunkBytes + ((n & 7) * 4 + (U & 3)) * 16;
+    const uint32_t byte = meta & 0xFFu;
+    const uint32_t base2 = byte * 0x00200020u + 0x26802680u;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int W = l + 2 * c;                             // this lane's code words
+      uint32_t r[4] = {0u, 0u, 0u, 0u};
+      if (n < M) {
+        if (byte == 0xFFu) r[0] = r[1] = r[2] = r[3] = 0x7FC07FC0u;
+        else decode_word_regs(meta, base2, W, codes[c], r);
+      }
+      *reinterpret_cast<uint4*>(dst + W * kTokChunkBytes) = make_uint4(r[0], r[1], r[2], r[3]);
+    }
+  }
+}
+
 // Per-unit part of the weight decode: the BF16 bits of E6M2 / 4 in both halves, the constant that is
 // OR-ed into every element pair (128.0, or NaN for a NaN unit, Eq. 2), and E1_8[j] + E1_16[2j] /
 // E1_16[2j+1] for all eight words as two-bit fields of the low / high half.
@@ -250,10 +320,13 @@ __device__ __forceinline__ bool wait_announced(const volatile int* slot, int kc,
   }
 }
 
-// Shared memory: [spread table 1 KB][partial sums][barriers, abort word, announced chunks: 384 B][ring of stages, 128-byte aligned]
-template <int kTokTiles, int kGemvWarps>
+// Shared memory: [spread table 1 KB][partial sums][barriers, abort word, announced chunks: 384 B][resident tokens (kSrc 1, 2)]
+// [ring of stages, 128-byte aligned]
+template <int kTokTiles, int kGemvWarps, int kSrc>
 __global__ void __launch_bounds__((kGemvWarps + 1) * 32, 1)
 gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__ CUtensorMap tm_short, const GemvParams p) {
+  constexpr bool kResident = kSrc != kSrcWorkspace;
+  static_assert(!kResident || kTokTiles == 1, "resident tokens: one n-tile");
   constexpr int kTokBytes = kTokTiles * kTileChunkBytes;
   constexpr int kRedBytes = kGemvWarps * 32 * 4 * kTokTiles * 4;     // partial accumulators of every consumer warp
   extern __shared__ uint8_t smem_raw[];
@@ -265,9 +338,11 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
   const uint32_t full = bar_base, empty = bar_base + 8 * kMaxStages;
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(gen_base + 1024 + kRedBytes + 16 * kMaxStages);
   volatile int* announced = reinterpret_cast<volatile int*>(gen_base + 1024 + kRedBytes + 16 * kMaxStages + 16);   // chunk in each stage
-  const uint32_t ring = bar_base + 384;
+  const uint32_t tok_res = bar_base + 384;                              // resident tokens: num_kc chunks of kTokBytes
+  uint8_t* tok_res_gen = gen_base + 1024 + kRedBytes + 384;
+  const uint32_t ring = tok_res + (kResident ? static_cast<uint32_t>(p.num_kc) * kTokBytes : 0u);
   const uint32_t w_bytes_max = static_cast<uint32_t>(p.max_blocks) * kBlockBytes;
-  const uint32_t stage_bytes = w_bytes_max + kTokBytes;
+  const uint32_t stage_bytes = w_bytes_max + (kResident ? 0 : kTokBytes);
 
   // this CTA's run of 8-row blocks
   const int64_t blk_begin = static_cast<int64_t>(blockIdx.x) * p.num_blocks / gridDim.x;
@@ -292,7 +367,7 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
     // ---------------------------------------------------------------- producer
     if (lane == 0) {
       const CUtensorMap* map = nblk == p.max_blocks ? &tm_full : &tm_short;
-      const uint32_t tx = static_cast<uint32_t>(nblk) * kBlockBytes + kTokBytes;
+      const uint32_t tx = static_cast<uint32_t>(nblk) * kBlockBytes + (kResident ? 0 : kTokBytes);
       const int row0 = static_cast<int>(blk_begin * kBlockRows);
       // Launched as a programmatic dependent of the token preparation: the weights of the first ring
       // of stages are requested first, then the preparation grid is waited for, then the tokens follow.
@@ -302,10 +377,12 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
         mbar_expect_tx(full + 8 * kc, tx);
         tma_load_2d(ring + kc * stage_bytes, map, kc * kRawRowBytes, row0, full + 8 * kc);
       }
-      asm volatile("griddepcontrol.wait;" ::: "memory");
-      for (int kc = 0; kc < head; ++kc)
-        bulk_load_1d(ring + kc * stage_bytes + w_bytes_max, p.tokens + static_cast<int64_t>(kc) * kTokBytes, kTokBytes,
-                     full + 8 * kc);
+      if (!kResident) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        for (int kc = 0; kc < head; ++kc)
+          bulk_load_1d(ring + kc * stage_bytes + w_bytes_max, p.tokens + static_cast<int64_t>(kc) * kTokBytes, kTokBytes,
+                       full + 8 * kc);
+      }
       uint32_t s = 0, ph = 1;                          // stage and phase of chunk `head`
       for (int kc = head; kc < p.num_kc; ++kc) {
         if (!mbar_wait(empty + 8 * s, ph ^ 1u, abort_flag, 32)) break;
@@ -314,7 +391,7 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
         mbar_expect_tx(full + 8 * s, tx);
         const uint32_t dst = ring + s * stage_bytes;
         tma_load_2d(dst, map, kc * kRawRowBytes, row0, full + 8 * s);
-        bulk_load_1d(dst + w_bytes_max, p.tokens + static_cast<int64_t>(kc) * kTokBytes, kTokBytes, full + 8 * s);
+        if (!kResident) bulk_load_1d(dst + w_bytes_max, p.tokens + static_cast<int64_t>(kc) * kTokBytes, kTokBytes, full + 8 * s);
         if (++s == static_cast<uint32_t>(p.stages)) { s = 0; ph ^= 1u; }
       }
     }
@@ -331,7 +408,15 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
       for (int i = 0; i < 4; ++i) acc[t][i] = 0.0f;
     const uint32_t off_lo = static_cast<uint32_t>(16 * pair + g) * kRawRowBytes + q * kUnitBytes;   // MMA row g
     const uint32_t off_hi = off_lo + 8 * kRawRowBytes;                                                // MMA row g + 8
-    const uint32_t off_tok = w_bytes_max + static_cast<uint32_t>(lane) * 16;
+    const uint32_t off_tok = (kResident ? 0u : w_bytes_max) + static_cast<uint32_t>(lane) * 16;
+    if (kResident) {
+      // every consumer thread helps to build the CTA's own copy of the tokens, then all of them meet
+      const int64_t upr = static_cast<int64_t>(p.num_kc) * kRawUnits;
+      if (kSrc == kSrcUnits) build_tokens_from_units(p.A, p.M, upr, tok_res_gen, threadIdx.x, kGemvWarps * 32);
+      else if (p.rha) build_tokens_from_bf16<true>(p.X, p.ld_x, p.M, upr, tok_res_gen, threadIdx.x, kGemvWarps * 32);
+      else build_tokens_from_bf16<false>(p.X, p.ld_x, p.M, upr, tok_res_gen, threadIdx.x, kGemvWarps * 32);
+      asm volatile("bar.sync 1, %0;" ::"n"(kGemvWarps * 32) : "memory");
+    }
     if (active) {
       uint32_t s = static_cast<uint32_t>(way % p.stages), ph = static_cast<uint32_t>(way / p.stages) & 1u;
       const uint32_t s_step = static_cast<uint32_t>(ways % p.stages), ph_step = static_cast<uint32_t>(ways / p.stages);
@@ -341,6 +426,7 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
                                                mbar_wait(full + 8 * s, ph, abort_flag))))
           break;
         const uint32_t st = ring + s * stage_bytes;
+        const uint32_t tk = kResident ? tok_res + static_cast<uint32_t>(kc) * kTokBytes : st;      // this chunk's tokens
         const uint32_t ml = lds32(st + off_lo), mh = has_hi ? lds32(st + off_hi) : 0u;
         const UnitPrep ul = prepare_unit(ml, lut), uh = prepare_unit(mh, lut);
         // a short loop rather than eight unrolled words: the body stays small enough for the instruction cache
@@ -348,7 +434,7 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
         for (int j = 0; j < 8; ++j) {
           uint4 x[kTokTiles];
 #pragma unroll
-          for (int t = 0; t < kTokTiles; ++t) x[t] = lds128(st + off_tok + (t * 8 + j) * kTokChunkBytes);
+          for (int t = 0; t < kTokTiles; ++t) x[t] = lds128(tk + off_tok + (t * 8 + j) * kTokChunkBytes);
           uint32_t a[4], b[4] = {0u, 0u, 0u, 0u};
           decode_word(ul, j, lds32(st + off_lo + 4 + 4 * j), p.mul, a);
           if (has_hi) decode_word(uh, j, lds32(st + off_hi + 4 + 4 * j), p.mul, b);
@@ -397,9 +483,11 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
   }
 }
 
-template <int kTokTiles, int kGemvWarps>
+template <int kTokTiles, int kGemvWarps, int kSrc = kSrcWorkspace>
 hif4_status launch_gemv_t(const void* B, int64_t upr, GemvParams p, cudaStream_t st) {
+  constexpr bool kResident = kSrc != kSrcWorkspace;
   constexpr int kTokBytes = kTokTiles * kTileChunkBytes;
+  const int resident_bytes = kResident ? p.num_kc * kTokBytes : 0;
   constexpr int kFixed = 128 + 1024 + kGemvWarps * 32 * 4 * kTokTiles * 4 + 384;
   // One CTA per SM (several rounds of them when a CTA would get more than kMaxBlocks blocks).
   const int64_t sms = sm_count();
@@ -407,13 +495,14 @@ hif4_status launch_gemv_t(const void* B, int64_t upr, GemvParams p, cudaStream_t
   const int64_t grid = p.num_blocks < sms * rounds ? p.num_blocks : sms * rounds;
   if (grid > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
   p.max_blocks = static_cast<int>(ceil_div64(p.num_blocks, grid));
-  const int stage_bytes = p.max_blocks * kBlockBytes + kTokBytes;
-  p.stages = kRingBudget / stage_bytes;
+  const int stage_bytes = p.max_blocks * kBlockBytes + (kResident ? 0 : kTokBytes);
+  p.stages = (kRingBudget - resident_bytes) / stage_bytes;
   if (p.stages > kMaxStages) p.stages = kMaxStages;
   if (p.stages > p.num_kc) p.stages = p.num_kc;
-  const int smem = kFixed + p.stages * stage_bytes;
+  if (p.stages < 1) return HIF4_ERR_SHAPE;
+  const int smem = kFixed + resident_bytes + p.stages * stage_bytes;
   static uint64_t smem_opt_in = 0;
-  if (!ensure_dynamic_smem(gemv_kernel<kTokTiles, kGemvWarps>, kFixed + kRingBudget, smem_opt_in)) return HIF4_ERR_CUDA;
+  if (!ensure_dynamic_smem(gemv_kernel<kTokTiles, kGemvWarps, kSrc>, kFixed + kRingBudget, smem_opt_in)) return HIF4_ERR_CUDA;
   CUtensorMap tm_full, tm_short;
   if (!make_unit_map(&tm_full, B, p.N, upr, p.max_blocks * kBlockRows)) return HIF4_ERR_CUDA;
   if (!make_unit_map(&tm_short, B, p.N, upr, (p.max_blocks > 1 ? p.max_blocks - 1 : 1) * kBlockRows)) return HIF4_ERR_CUDA;
@@ -427,7 +516,7 @@ hif4_status launch_gemv_t(const void* B, int64_t upr, GemvParams p, cudaStream_t
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, gemv_kernel<kTokTiles, kGemvWarps>, tm_full, tm_short, p) != cudaSuccess) {
+  if (cudaLaunchKernelEx(&cfg, gemv_kernel<kTokTiles, kGemvWarps, kSrc>, tm_full, tm_short, p) != cudaSuccess) {
     (void)cudaGetLastError();
     return HIF4_ERR_CUDA;
   }
@@ -461,6 +550,16 @@ bool gemv_params(GemvParams& p, float* C, int64_t M, int64_t N, int64_t K, int64
   p.error_word = device_error_word();
   return true;
 }
+// One n-tile of tokens and a K short enough for the tokens to stay in shared memory: the streaming kernel builds them itself.
+bool gemv_tokens_fit_resident(int m_pad, int num_kc) { return m_pad == 8 && num_kc * kTileChunkBytes <= kResidentMaxBytes; }
+template <int kSrc>
+hif4_status launch_gemv_resident(const void* B, const GemvParams& p, int64_t upr, cudaStream_t st) {
+  const int64_t sms = sm_count();
+  const int64_t rounds = ceil_div64(p.num_blocks, sms * kMaxBlocks);
+  const int64_t grid = p.num_blocks < sms * rounds ? p.num_blocks : sms * rounds;
+  const bool many = ceil_div64(p.num_blocks, grid) >= 9;
+  return many ? launch_gemv_t<1, kGemvWarpsMany, kSrc>(B, upr, p, st) : launch_gemv_t<1, kGemvWarpsFew, kSrc>(B, upr, p, st);
+}
 // The streaming kernel on tokens that the preceding launch in `st` has prepared.
 hif4_status launch_gemv_stream(const void* B, const GemvParams& p, int m_pad, int64_t upr, cudaStream_t st) {
   // blocks of the largest CTA (same arithmetic as launch_gemv_t): nine or more are five row pairs or more
@@ -482,6 +581,7 @@ hif4_status launch_gemv(const void* A, const void* B, float* C, int64_t M, int64
   if (!p.error_word) return HIF4_ERR_CUDA;
   const int m_pad = static_cast<int>(gemv_m_pad(M));
   const int64_t upr = K / kUnitElems;
+  if (gemv_tokens_fit_resident(m_pad, p.num_kc)) return launch_gemv_resident<kSrcUnits>(B, p, upr, st);     // one launch
   const int64_t prep = static_cast<int64_t>(m_pad) * upr;
   gemv_prepare_tokens_kernel<<<static_cast<unsigned>(ceil_div64(prep, 128)), 128, 0, st>>>(p.A, p.M, m_pad, upr, p.tokens);
   note_launch();
@@ -502,6 +602,10 @@ hif4_status launch_gemv_linear(const void* X, hif4_dtype dt, int64_t ld_x, int r
   if (!p.error_word) return HIF4_ERR_CUDA;
   const int m_pad = static_cast<int>(gemv_m_pad(M));
   const int64_t upr = K / kUnitElems;
+  if (dt == HIF4_BF16 && gemv_tokens_fit_resident(m_pad, p.num_kc)) {        // one launch: conversion, decode and streaming
+    p.X = static_cast<const uint16_t*>(X); p.ld_x = ld_x; p.rha = rha;
+    return launch_gemv_resident<kSrcBf16>(B, p, upr, st);
+  }
   const int lanes = dt == HIF4_BF16 ? 2 : 4;             // lanes per unit of the encoder
   const unsigned blocks = static_cast<unsigned>(ceil_div64(lanes * static_cast<int64_t>(m_pad) * upr, 128));
   if (dt == HIF4_BF16) {

@@ -158,7 +158,8 @@ def test_llama_decode_linears_replayed_from_a_cuda_graph(hif4):
     before = hif4.launch_count()
     with torch.cuda.graph(graph):
         run()
-    assert hif4.launch_count() - before == 2 * len(shapes), "token preparation + streaming kernel per linear"
+    want_launches = sum(1 if (M <= 8 and K <= 6144) else 2 for (M, K, N) in shapes)
+    assert hif4.launch_count() - before == want_launches, "streaming kernel per linear, preceded by a token kernel for M = 16 or long K"
     for c in cs.values():
         c.fill_(-7.0)
     for _ in range(3):

@@ -349,7 +349,8 @@ def gemv_path(hif4):
 @pytest.mark.parametrize("M,N,K", [(1, 1, 256), (1, 64, 256), (2, 33, 512), (7, 200, 1024), (8, 4096, 256), (9, 130, 768),
                                    (16, 1000, 2304), (16, 64, 4096), (5, 9475, 256), (3, 31, 5120), (12, 77, 14336),
                                    (1, 40003, 256), (16, 2376, 1024), (10, 1192, 512), (4, 19000, 256),
-                                   (17, 300, 256), (32, 1000, 1024), (25, 4200, 512), (31, 77, 4096), (20, 14336, 256)])
+                                   (17, 300, 256), (32, 1000, 1024), (25, 4200, 512), (31, 77, 4096), (20, 14336, 256),
+                                   (8, 300, 6144), (8, 300, 6400), (5, 14336, 4096), (1, 1030, 4096)])
 def test_weight_streaming_kernel_full_compare(gemv_path, M, N, K):
     hif4 = gemv_path
     g = torch.Generator(device="cuda"); g.manual_seed(M * 11 + N)
@@ -359,7 +360,8 @@ def test_weight_streaming_kernel_full_compare(gemv_path, M, N, K):
     before = hif4.launch_count()
     out = torch.full((M + 2, N + 3), -5.0, dtype=torch.float32, device="cuda")
     C = check_full(hif4, a, b, f"gemv {M}x{N}x{K}", out=out[1:M + 1, 1:N + 1])
-    assert hif4.launch_count() - before == 2, "token preparation + streaming kernel"
+    one_launch = M <= 8 and K <= 6144            # few tokens, short K: the streaming kernel decodes the tokens itself
+    assert hif4.launch_count() - before == (1 if one_launch else 2), "token preparation + streaming kernel, or the latter alone"
     assert (out[0] == -5.0).all() and (out[M + 1] == -5.0).all() and (out[:, 0] == -5.0).all() and (out[:, N + 1:] == -5.0).all()
     C2 = hif4.hif4_gemm(a, b)
     assert torch.equal(C.contiguous(), C2), "two runs of the weight-streaming kernel differ"
@@ -475,8 +477,9 @@ def test_linear_is_quantize_then_gemm(hif4, M, N, K, dtype):
                                    (24, 520, 1024), (32, 64, 256)])
 def test_linear_with_few_rows_quantizes_inside_the_token_preparation(hif4, M, N, K, dtype, mode):
     """M <= 32 rows of activations: hif4_linear runs two kernels (quantize-and-decode of the tokens, weight
-    streaming) instead of three and gives exactly the bits of hif4_quantize followed by hif4_gemm -- on a strided
-    source with spikes, a NaN and an Inf, for every source type and both rounding modes."""
+    streaming) instead of three -- a single one for up to eight BF16 rows and K <= 6144 -- and gives exactly the bits
+    of hif4_quantize followed by hif4_gemm, on a strided source with spikes, a NaN and an Inf, for every source type
+    and both rounding modes."""
     g = torch.Generator(device="cuda"); g.manual_seed(M * 3 + N + K + mode)
     wide = torch.randn(M, K + 64, generator=g, device="cuda").to(dtype)
     x = wide[:, 64:]                                      # row stride K + 64
@@ -487,7 +490,8 @@ def test_linear_with_few_rows_quantizes_inside_the_token_preparation(hif4, M, N,
     w = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
     before = hif4.launch_count()
     y = hif4.hif4_linear(x, w, mode=mode)
-    assert hif4.launch_count() - before == 2
+    one_launch = M <= 8 and K <= 6144 and dtype == torch.bfloat16     # conversion, token decode and streaming in one kernel
+    assert hif4.launch_count() - before == (1 if one_launch else 2)
     want = hif4.hif4_gemm(hif4.hif4_quantize(x, mode), w)
     assert torch.equal(y.view(torch.int32), want.view(torch.int32)), "fused token preparation differs from quantize + GEMM"
     assert hif4.hif4_last_device_status() == 0
