@@ -60,14 +60,14 @@ typedef enum {
   HIF4_ERR_UNSUPPORTED = 8     /* valid request that this build does not implement             */
 } hif4_status;
 
-/* HIF4_FP16 is a source type only (hif4_quantize, hif4_linear): Section II-B applies the conversion to
- * "other high-precision formats, such as FP32 and FP16"; FP16 arithmetic cannot hold the reciprocal of an
+/* HIF4_FP16 is a source type only (hif4_quantize, hif4_linear): Section II-B extends the conversion to
+ * further source types and names FP32 and FP16; FP16 arithmetic cannot hold the reciprocal of an
  * E6M2 scale (up to 2^48), so FP16 elements are widened exactly to FP32 and Algorithm 1 runs in FP32
  * arithmetic.  hif4_dequantize returns HIF4_ERR_DTYPE for it (HiF4's range exceeds FP16's).  */
 typedef enum { HIF4_BF16 = 0, HIF4_FP32 = 1, HIF4_FP16 = 2 } hif4_dtype;
 
-/* Rounding used where Algorithm 1 rounds to E6M2 and to S1P2 ("round-half-to-even or
- * round-half-away-from-zero", Section II-B).  Products inside the algorithm always round to
+/* Rounding used where Algorithm 1 rounds to E6M2 and to S1P2 (Section II-B allows half-to-even or
+ * half-away-from-zero).  Products inside the algorithm always round to
  * nearest-even.  */
 typedef enum { HIF4_RNE = 0, HIF4_RHA = 1 } hif4_round;
 
@@ -89,8 +89,8 @@ hif4_status hif4_quantize(const void* src, hif4_dtype dt, int64_t rows, int64_t 
 
 /* hif4_quantize_transposed -- the same conversion with the units running down the columns: unit r of
  * column c holds src[64 r .. 64 r + 63][c], i.e. dst is hif4_quantize of the transposed matrix without the
- * transpose ever being written.  (Algorithm 1 converts "a vector of 64" values and does not say how the
- * vector lies in memory; Eq. 3 needs both GEMM operands cut along the contraction dimension, so a matrix
+ * transpose ever being written.  (Algorithm 1 converts 64 values at a time and does not say how those
+ * 64 lie in memory; Eq. 3 needs both GEMM operands cut along the contraction dimension, so a matrix
  * that is contracted along its rows -- a weight kept as [K, N], or any operand of a transposed product --
  * is quantized this way.)
  *   src        device, [rows, cols] of `dt` (any source type of hif4_quantize, same working precision), row

@@ -115,7 +115,7 @@ def round_to(v: float, dt: int) -> float:
 def quantize(src: np.ndarray, mode: int = RNE, nthreads: int = 1) -> np.ndarray:
     """Algorithm 1 on a 2-D array: ``uint16`` = BF16 bit patterns, ``float32`` = FP32, ``float16`` = FP16.
 
-    Section II-B extends the conversion to "FP32 and FP16" sources without further detail.  FP16 arithmetic
+    Section II-B extends the conversion to FP32 and FP16 sources without further detail.  FP16 arithmetic
     cannot hold the reciprocal of an E6M2 scale (up to 2^48), so an FP16 source is read as: widen every
     element to FP32 (a storage conversion, exact) and run the FP32 form of Algorithm 1."""
     assert src.ndim == 2 and src.shape[1] % UNIT_ELEMS == 0

@@ -22,7 +22,7 @@
 // product, table entry or threshold product would change a byte, a micro-exponent or a code.
 // Parity unpinned: the byte/bit order inside a unit and the choice of FP32 working precision for
 // FP32/FP16 sources are conventions of this repository (the paper's unit figure is not available
-// as text and it only says that "a similar procedure" applies to those types); the paper prints no
+// as text and it only says that those types are converted in a like manner); the paper prints no
 // worked encoding, so the worked examples are derived by hand from Algorithm 1.
 
 #include <cmath>
@@ -443,7 +443,7 @@ double hif4_ref_best_unit(const double* x, void* best_unit) {
 //   E2M1 element: magnitudes {0, 0.5, 1, 1.5, 2, 3, 4, 6}, round to nearest, ties to the even code, saturating.
 //   MXFP4: blocks of 32, power-of-two scale 2^(floor(log2 amax) - 2) (2 = the largest E2M1 exponent), exponent
 //          clamped to [-127, 127]; elements round(x / scale), so values between 6 and 8 scales saturate to 6.
-//   NVFP4: blocks of 16, scale = E4M3(amax / 6) ("normalize the peak magnitude of each group to 6"), elements
+//   NVFP4: blocks of 16, scale = E4M3(amax / 6) (the group's peak lands on 6, the largest E2M1 magnitude), elements
 //          round(x / scale).  With per-tensor scaling the tensor is first multiplied by gain = 2688 / max|x|
 //          (2688 = 448 * 6) and the result divided by the gain again.
 namespace {
