@@ -160,7 +160,7 @@ def test_worked_example_fp32_source():
 
 
 def test_worked_examples_fp16_source():
-    """FP16 source (Section II-B: "FP32 and FP16"): elements are widened to FP32 and Algorithm 1 runs in FP32
+    """FP16 source (Section II-B names FP32 and FP16 as further source types): elements are widened to FP32 and Algorithm 1 runs in FP32
     arithmetic.  Hand cases: the FP32 example above with FP16 storage, where x8 = fp16(0.0585) =
     0.058502197265625: 0.0585022 * 6.4000001 = 0.374414 -> 1.49766 quarters -> code 1 (narrowing the source
     to BF16 instead would give 0.05859375 and the tie code 2); the smallest FP16 subnormal 2^-24:
