@@ -148,6 +148,15 @@ def test_grouped_gemm_with_empty_and_ragged_groups(hif4):
     _grouped_case(hif4, [200], N=130, K=512, seed=33)
 
 
+def test_grouped_gemm_small_and_large_token_tiles_odd_weight_tile_count(hif4):
+    """Token tiles of at most 64 rows take two weight tiles per work record, larger ones one: groups on both sides of
+    that limit (64 / 65 rows, a 256 + 40 row group whose last tile is small, single rows, empty groups), with three
+    weight tiles (the last record of a small tile has no second weight tile and must not touch the next group's rows)
+    and with four, over several K chunks.  Every entry against the oracle; the guard value around C stays."""
+    for (N, K, seed) in ((700, 768, 51), (1024, 512, 52), (257, 256, 53)):
+        _grouped_case(hif4, [64, 65, 0, 296, 1, 33, 0, 130, 32], N=N, K=K, seed=seed)
+
+
 def test_grouped_gemm_moe_routing_sampled(hif4):
     r = wl.moe_routing(tokens=512, experts=32, topk=4, device="cuda")
     off = r["offsets"]
