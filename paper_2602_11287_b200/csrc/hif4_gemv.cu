@@ -372,6 +372,9 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
       // Launched as a programmatic dependent of the token preparation: the weights of the first ring
       // of stages are requested first, then the preparation grid is waited for, then the tokens follow.
       const int head = p.num_kc < p.stages ? p.num_kc : p.stages;
+      // With resident tokens the preceding launch in the stream is the caller's (it may have written the weights, the
+      // tokens, or still read C): the CTA may be scheduled early, but nothing is read or written before that grid is done.
+      if (kResident) asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int kc = 0; kc < head; ++kc) {
         announced[kc] = kc;
         mbar_expect_tx(full + 8 * kc, tx);
@@ -410,6 +413,7 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
     const uint32_t off_hi = off_lo + 8 * kRawRowBytes;                                                // MMA row g + 8
     const uint32_t off_tok = (kResident ? 0u : w_bytes_max) + static_cast<uint32_t>(lane) * 16;
     if (kResident) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");      // see the producer
       // every consumer thread helps to build the CTA's own copy of the tokens, then all of them meet
       const int64_t upr = static_cast<int64_t>(p.num_kc) * kRawUnits;
       if (kSrc == kSrcUnits) build_tokens_from_units(p.A, p.M, upr, tok_res_gen, threadIdx.x, kGemvWarps * 32);
