@@ -552,6 +552,32 @@ def measure_per_config(hif4, dev, peaks, sampler, matmul_floor):
                         "paper": "HiF4 : NVFP4 : MXFP4 = 1 : 1.32 : 1.89", "mean_nvfp4_pts": round(statistics.mean(r["nvfp4_pts"] for r in study), 4),
                         "mean_mxfp4": round(statistics.mean(r["mxfp4"] for r in study), 4), "rows": study,
                         "us_per_1024x1024_matrix": us}
+    # ---- the two variants kept behind the test hook, against the default kernels on one shape each
+    variants = {}
+    try:
+        M, N, K = 1, 14336, 4096                     # Eq. 3's factorisation on FP8 operands (path 5) vs the BF16-folded form
+        a = hif4.hif4_quantize(wl.llama_activations(M, K, device=dev))
+        wq = hif4.hif4_quantize(wl.gaussian(N, K, 0.02, seed=5, device=dev))
+        c = torch.empty(M, N, dtype=torch.float32, device=dev)
+        ws = torch.empty(max(hif4.hif4_gemm_workspace(M, N, K), 256), dtype=torch.uint8, device=dev)
+        row = {"shape": {"M": M, "N": N, "K": K}, "timing": "20 launches back to back, L2 warm (33 MB of weights)"}
+        for name, path in (("bf16_folded_default_us", 0), ("fp8_operands_eq3_scaling_us", 5)):
+            hif4.hif4_debug_set_gemm_path(path)
+            row[name] = round(_timed(lambda: hif4.hif4_gemm(a, wq, out=c, workspace=ws), 20, sampler)[0], 2)
+        variants["weight_streaming_fp8_operands"] = row
+        M, N, K = 4096, 1024, 4096                   # activation conversion inside the pair kernel (path 6) vs two launches
+        x = wl.llama_activations(M, K, device=dev)
+        wq = hif4.hif4_quantize(wl.gaussian(N, K, 0.02, seed=6, device=dev))
+        y = torch.empty(M, N, dtype=torch.float32, device=dev)
+        ws = torch.empty(max(hif4.hif4_linear_workspace(M, N, K), 256), dtype=torch.uint8, device=dev)
+        row = {"shape": {"M": M, "N": N, "K": K}, "timing": "20 calls of hif4_linear back to back"}
+        for name, path in (("quantize_then_gemm_default_us", 0), ("conversion_inside_the_gemm_us", 6)):
+            hif4.hif4_debug_set_gemm_path(path)
+            row[name] = round(_timed(lambda: hif4.hif4_linear(x, wq, out=y, workspace=ws), 20, sampler)[0], 2)
+        variants["linear_fused_conversion"] = row
+    finally:
+        hif4.hif4_debug_set_gemm_path(0)
+    out["variants_behind_the_test_hook"] = variants
     status = hif4.hif4_last_device_status()
     if status != 0:
         raise SystemExit(f"device status {status}: {hif4.status_string(status)}")

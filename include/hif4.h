@@ -224,8 +224,10 @@ const char* hif4_status_string(hif4_status s);
  * hif4_debug_set_gemm_path: 0 = choose the GEMM kernel by shape (default), 1 = CUDA-core kernel only,
  * 2 = the single-CTA tensor-core (tcgen05) kernel whenever it is legal (K % 256 == 0, 16-byte aligned
  * operands), even for small M, 3 = the CTA-pair tensor-core kernel (256 x 256 tiles) whenever it is legal,
- * 4 = the weight-streaming kernel whenever it is legal (M <= 32), 6 = hif4_linear converts BF16 activations inside
- * the CTA-pair kernel whenever that is legal (M > 128).  Process-wide and not thread-safe.
+ * 4 = the weight-streaming kernel whenever it is legal (M <= 32), 5 = the variant of that kernel that follows
+ * Eq. 3's factorisation (FP8 E4M3 tensor-core operands holding the elements with their micro-exponents, the two
+ * level-1 scales applied to each unit pair's sum) whenever it is legal (M <= 32), 6 = hif4_linear converts BF16
+ * activations inside the CTA-pair kernel whenever that is legal (M > 128).  Process-wide and not thread-safe.
  * hif4_gemm_workspace does not depend on it: it always reports the largest need over all paths.
  *
  * hif4_debug_launch_count: number of kernels this library has launched in this process (monotonic,

@@ -7,8 +7,9 @@ using namespace hif4;
 namespace {
 // Test hook (hif4_debug_set_gemm_path): 0 = choose by shape, 1 = CUDA-core kernel only, 2 = single-CTA
 // tensor-core kernel whenever it is legal, 3 = CTA-pair tensor-core kernel whenever it is legal,
-// 4 = weight-streaming kernel whenever it is legal (M <= kGemvMaxM), 6 = hif4_linear converts BF16 activations inside
-// the CTA-pair kernel whenever that is legal (hif4_gemm itself behaves as under 0).
+// 4 = weight-streaming kernel whenever it is legal (M <= kGemvMaxM), 5 = the weight-streaming kernel on FP8 operands
+// with Eq. 3's per-unit-pair scaling whenever it is legal (same shapes), 6 = hif4_linear converts BF16 activations
+// inside the CTA-pair kernel whenever that is legal (hif4_gemm itself behaves as under 0).
 int g_gemm_path = 0;
 constexpr int64_t kPairMinM = 129;      // below that a 256-row pair tile would be half empty
 constexpr int64_t kFuseMaxColumnTiles = 0;   // hif4_linear: in-kernel conversion for C with at most this many 256-column tiles
@@ -33,6 +34,7 @@ extern "C" hif4_status hif4_gemm_workspace(int64_t M, int64_t N, int64_t K, size
   // time: decoded tokens of the weight-streaming path (M <= kGemvMaxM), completion words of the K slices of
   // the swapped pair kernel (few rows) and of the tiles that the pair kernel shares along K.
   *bytes = gemv_workspace_bytes(M, K);
+  if (gemv8_workspace_bytes(M, K) > *bytes) *bytes = gemv8_workspace_bytes(M, K);
   if (M > kGemvMaxM && M < kPairMinM) {
     const size_t few_bytes = gemm_tc2_swapped_workspace_bytes(M, N, K);
     if (few_bytes > *bytes) *bytes = few_bytes;
@@ -64,6 +66,11 @@ extern "C" hif4_status hif4_gemm(const void* A_units, const void* B_units, float
     if (!workspace || workspace_bytes < gemv_workspace_bytes(M, K)) return HIF4_ERR_WORKSPACE;
     if (!aligned(workspace, 256)) return HIF4_ERR_ALIGN;
     return launch_gemv(A_units, B_units, C, M, N, K, ldc, workspace, st);
+  }
+  if (g_gemm_path == 5 && gemv_supported(A_units, B_units, M, N, K)) {
+    if (!workspace || workspace_bytes < gemv8_workspace_bytes(M, K)) return HIF4_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return HIF4_ERR_ALIGN;
+    return launch_gemv8(A_units, B_units, C, M, N, K, ldc, workspace, st);
   }
   const bool tc_ok = g_gemm_path != 1 && gemm_tc_supported(A_units, B_units, M, N, N, K);
   if (tc_ok && g_gemm_path != 2 && (g_gemm_path == 3 || M >= kPairMinM) && gemm_tc2_supported(A_units, B_units, M, N, K)) {

@@ -37,6 +37,13 @@ hif4_status launch_gemv(const void* A, const void* B, float* C, int64_t M, int64
 bool gemv_linear_supported(const void* X, hif4_dtype dt, int64_t ld_x, const void* B, int64_t M, int64_t N, int64_t K);
 hif4_status launch_gemv_linear(const void* X, hif4_dtype dt, int64_t ld_x, int rha, const void* B, float* C, int64_t M,
                                int64_t N, int64_t K, int64_t ldc, void* workspace, cudaStream_t st);
+// The weight-streaming path on Eq. 3's factorisation: E4M3 operands that hold the elements with their micro-exponents,
+// the two level-1 scales applied to the FP32 sum of each unit pair.  Same requirements as the path above; workspace
+// of gemv8_workspace_bytes (the tokens as E4M3 operand bytes and per-unit scales).  Slower than the BF16 form on
+// sm_100a (the legacy FP8 mma.sync has no native path there); reachable through the test hook only.
+size_t gemv8_workspace_bytes(int64_t M, int64_t K);
+hif4_status launch_gemv8(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t ldc,
+                         void* workspace, cudaStream_t st);
 size_t grouped_tc_workspace_bytes(int num_groups, int64_t total_rows);
 hif4_status launch_grouped_gemm_tc(const void* A, const void* B, float* C, const int64_t* offsets, int num_groups,
                                    int64_t total_rows, int64_t N, int64_t K, int64_t ldc, void* workspace,

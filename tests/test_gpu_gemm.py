@@ -393,6 +393,50 @@ def test_weight_streaming_kernel_random_units_and_nan(gemv_path):
     assert np.all(np.abs(got - ref)[~nan] <= TOL * refabs[~nan] + 1e-300)
 
 
+@pytest.fixture()
+def fp8_path(hif4):
+    """5 = the weight-streaming kernel on Eq. 3's factorisation: E4M3 operands, level-1 scales per unit pair."""
+    hif4.hif4_debug_set_gemm_path(5)
+    yield hif4
+    hif4.hif4_debug_set_gemm_path(0)
+    assert hif4.hif4_last_device_status() == 0, "a bounded wait inside the kernel ran out"
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 1, 256), (2, 33, 512), (7, 200, 1024), (8, 4096, 256), (9, 130, 768), (16, 1000, 2304),
+                                   (3, 31, 5120), (12, 77, 14336), (1, 40003, 256), (17, 300, 256), (32, 1000, 1024),
+                                   (25, 4200, 512), (5, 14336, 4096)])
+def test_fp8_operand_kernel_full_compare(fp8_path, M, N, K):
+    """Section III-B's flow (small signed operands, one scale product per unit pair) on tensor-core FP8 operands gives
+    the product within the same tolerance as the kernels that fold the level-1 scale into BF16 operands."""
+    hif4 = fp8_path
+    g = torch.Generator(device="cuda"); g.manual_seed(M * 11 + N)
+    a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
+    b = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
+    before = hif4.launch_count()
+    out = torch.full((M + 2, N + 3), -5.0, dtype=torch.float32, device="cuda")
+    C = check_full(hif4, a, b, f"fp8 gemv {M}x{N}x{K}", out=out[1:M + 1, 1:N + 1])
+    assert hif4.launch_count() - before == 2, "token preparation + streaming kernel"
+    assert (out[0] == -5.0).all() and (out[M + 1] == -5.0).all() and (out[:, 0] == -5.0).all() and (out[:, N + 1:] == -5.0).all()
+    assert torch.equal(C.contiguous(), hif4.hif4_gemm(a, b)), "two runs differ"
+
+
+def test_fp8_operand_kernel_random_units_and_nan(fp8_path):
+    hif4 = fp8_path
+    rng = np.random.default_rng(82)
+    M, N, upr = 11, 150, 8
+    A = rng.integers(0, 256, (M, upr, 36), dtype=np.uint8)
+    B = rng.integers(0, 256, (N, upr, 36), dtype=np.uint8)
+    A[..., 0] = rng.integers(0x00, 0xFF, (M, upr)); B[..., 0] = rng.integers(0x40, 0xC0, (N, upr))
+    A[3, 5, 0] = 0xFF
+    B[149, 0, 0] = 0xFF
+    C = hif4.hif4_gemm(torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda())
+    ref, refabs = oracle.gemm_f64(A, B, nthreads=8)
+    got = C.cpu().numpy().astype(np.float64)
+    nan = np.isnan(ref)
+    assert nan[3].all() and nan[:, 149].all() and np.array_equal(np.isnan(got), nan)
+    assert np.all(np.abs(got - ref)[~nan] <= TOL * refabs[~nan] + 1e-300)
+
+
 def test_weight_streaming_kernel_needs_its_workspace(gemv_path):
     hif4 = gemv_path
     a = torch.zeros(4, 4, 36, dtype=torch.uint8, device="cuda")
@@ -435,7 +479,7 @@ def _one_hot_units(K):
     return B
 
 
-@pytest.mark.parametrize("path,rows", [(1, 510), (2, 510), (3, 510), (0, 100), (4, 16), (4, 7)])
+@pytest.mark.parametrize("path,rows", [(1, 510), (2, 510), (3, 510), (0, 100), (4, 16), (4, 7), (5, 16), (5, 7)])
 def test_every_code_under_every_scale_passes_through_the_gemm_exactly(hif4, path, rows):
     """C = A * B^T with one-hot rows in B returns the decoded elements of A themselves: each in-kernel
     decoder (CUDA cores, single CTA, CTA pair, swapped pair for few rows, weight streaming) must give
@@ -454,7 +498,7 @@ def test_every_code_under_every_scale_passes_through_the_gemm_exactly(hif4, path
             assert np.array_equal(got.view(np.uint32) & 0x7FFFFFFF, want_all[start:start + rows].view(np.uint32) & 0x7FFFFFFF)
             nz = want_all[start:start + rows] != 0                           # sign of zero products is not defined by Eq. 3
             assert np.array_equal(np.signbit(got)[nz], np.signbit(want_all[start:start + rows])[nz])
-            if path == 4:                                                    # (the streaming kernel takes M <= 16 only)
+            if path in (4, 5):                                               # (the streaming kernels take few rows only)
                 continue
             got_t = hif4.hif4_gemm(b, a).cpu().numpy()                     # and as the B operand
             assert np.array_equal(np.abs(got_t.T), np.abs(want_all[start:start + rows]))
@@ -567,7 +611,7 @@ def test_gemm_workspace_is_valid_under_every_path_override(hif4):
             need = hif4.hif4_gemm_workspace(M, N, K)
             ws = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
             ref, refabs = oracle.gemm_f64(a.cpu().numpy(), b.cpu().numpy(), nthreads=8)
-            for path in (0, 1, 2, 3, 4):
+            for path in (0, 1, 2, 3, 4, 5):
                 hif4.hif4_debug_set_gemm_path(path)
                 assert hif4.hif4_gemm_workspace(M, N, K) == need
                 c = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
