@@ -272,14 +272,19 @@ def run_cuda(args):
             graph_launches += hif4.launch_count() - n0
         torch.cuda.synchronize()
 
+    # NVTX ranges (visible to a timeline profiler; free otherwise) name the four parts of a step
+    group_names = ("decode linears M=1", "prefill linears 1-2", "decode linears M=16", "prefill linears 3-4")
+
     def step(events=None):
         for gi, shapes in enumerate(groups):
+            torch.cuda.nvtx.range_push(group_names[gi])
             if gi in graphs:
                 graphs[gi].replay()
             elif gi in (0, 2):
                 run_linears(shapes)
             else:
                 run_shapes(shapes, events)
+            torch.cuda.nvtx.range_pop()
 
     step()
     barrier()
@@ -289,8 +294,10 @@ def run_cuda(args):
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     host_t0 = time.time()
     t_start.record(stream)
+    torch.cuda.nvtx.range_push("timed steps")
     for _ in range(args.steps):
         step(events)
+    torch.cuda.nvtx.range_pop()
     t_end.record(stream)
     barrier()
     host_t1 = time.time()
