@@ -14,10 +14,12 @@
 //      decodes word after word straight into the A fragments (k slots 2q, 2q+1, 2q+8, 2q+9 of every MMA
 //      come from unit q on both operands, so the K order is permuted the same way on both sides).
 //      The K slices of a pair are summed through shared memory in a fixed order.
-//   3. Up to eight tokens and K <= 6144 (kSrc 1, 2): no token kernel at all.  Every CTA decodes the few tokens itself
-//      (from packed units, or from BF16 activations that it first converts with Algorithm 1) into a resident block of
-//      shared memory before its main loop, while its producer warp is already streaming weights; one launch per
-//      product instead of two, which is most of the time of the small shapes.
+//   3. Up to 16 tokens with few elements in all (kSrc 1, 2): no token kernel at all.  Every CTA decodes the few tokens
+//      itself (from packed units, or from BF16 activations that it first converts with Algorithm 1) into a resident
+//      block of shared memory before its main loop, while its producer warp is already streaming weights; one launch
+//      per product instead of two, which is most of the time of the small shapes.  The resident block keeps 1, 2, 4 or
+//      8 token rows per n-tile (the MMA lanes of the rows it leaves out read zeros); rows kept x K is limited to what
+//      a CTA builds in less time than the second launch costs (one token from packed units: K up to 49152).
 // Results are deterministic (no atomics).  Every mbarrier wait is bounded.
 #include "hif4_common.cuh"
 #include "hif4_gemm_internal.cuh"
@@ -39,7 +41,7 @@ constexpr int kGemvWarpsMany = 31, kGemvWarpsFew = 24;
 constexpr int kRingBudget = 176 * 1024;              // bytes of shared memory given to the ring of stages
 
 constexpr int kSrcWorkspace = 0, kSrcUnits = 1, kSrcBf16 = 2;   // where the streaming kernel gets its tokens from
-constexpr int kResidentMaxBytes = 96 * 1024;          // resident tokens: K / 256 chunks of 4 KB (one n-tile)
+constexpr int kResidentMaxBytes = 128 * 1024;         // resident tokens: K / 256 chunks of (n-tiles x 8 words x rows x 64) bytes
 
 struct GemvParams {
   const uint32_t* A;        // [M, K/64] units (tokens)
@@ -55,6 +57,7 @@ struct GemvParams {
   int num_blocks;           // ceil(N / 8)
   int max_blocks;           // 8-row blocks of the largest CTA; the others have one fewer
   int stages;
+  int res_rows;             // resident tokens: token rows kept per n-tile (1, 2, 4 or 8)
   DecodeMul mul;
   unsigned int* error_word;
 };
@@ -213,17 +216,20 @@ gemv_quantize_tokens32_kernel(const Src* __restrict__ X, int64_t ld_x, int M, in
   }
 }
 
-// Resident tokens (one n-tile of eight tokens, all K): the consumer warps of a CTA build them before the main loop.
-// From packed units: task (token n, unit U).
+// Resident tokens (`tiles` n-tiles of `rows` token rows each, all K): the consumer warps of a CTA build them before the
+// main loop.  Layout: chunk, n-tile, word W: rows x 4 units x 16 bytes, so that lane (token g, unit q) of a warp reads
+// at g * 64 + q * 16 of the word's line (lanes with g >= rows read nothing).  From packed units: task (token n, unit U).
 __device__ __forceinline__ void build_tokens_from_units(const uint32_t* __restrict__ A, int M, int64_t upr, uint8_t* tok,
-                                                        int tid, int nthreads) {
-  for (int64_t idx = tid; idx < 8 * upr; idx += nthreads) {
+                                                        int tiles, int rows, int tid, int nthreads) {
+  const int word_bytes = rows * 64;
+  for (int64_t idx = tid; idx < static_cast<int64_t>(tiles) * rows * upr; idx += nthreads) {
     const int n = static_cast<int>(idx / upr);
     const int64_t U = idx - static_cast<int64_t>(n) * upr;
-    uint8_t* dst = tok + ((U >> 2) * 8) * kTokChunkBytes + ((n & 7) * 4 + (U & 3)) * 16;
+    const int t = n / rows, row = n - t * rows;
+    uint8_t* dst = tok + (((U >> 2) * tiles + t) * 8) * word_bytes + (row * 4 + (U & 3)) * 16;
     if (n >= M) {
 #pragma unroll
-      for (int W = 0; W < 8; ++W) *reinterpret_cast<uint4*>(dst + W * kTokChunkBytes) = make_uint4(0u, 0u, 0u, 0u);
+      for (int W = 0; W < 8; ++W) *reinterpret_cast<uint4*>(dst + W * word_bytes) = make_uint4(0u, 0u, 0u, 0u);
       continue;
     }
     const uint32_t* unit = A + (static_cast<int64_t>(n) * upr + U) * kUnitWords;
@@ -232,21 +238,26 @@ __device__ __forceinline__ void build_tokens_from_units(const uint32_t* __restri
     for (int W = 0; W < 8; W += 2) {
       uint32_t r[8];
       decode_two_words(meta, W, __ldg(unit + 1 + W), __ldg(unit + 2 + W), r);
-      *reinterpret_cast<uint4*>(dst + W * kTokChunkBytes) = make_uint4(r[0], r[1], r[2], r[3]);
-      *reinterpret_cast<uint4*>(dst + (W + 1) * kTokChunkBytes) = make_uint4(r[4], r[5], r[6], r[7]);
+      *reinterpret_cast<uint4*>(dst + W * word_bytes) = make_uint4(r[0], r[1], r[2], r[3]);
+      *reinterpret_cast<uint4*>(dst + (W + 1) * word_bytes) = make_uint4(r[4], r[5], r[6], r[7]);
     }
   }
 }
 // From BF16 activations: Algorithm 1 with two lanes per unit (the streaming quantizer's own code), then Eq. 2 of the
-// unit just encoded.  Whole warps take part: 16 * upr lane tasks, a multiple of 32.
+// unit just encoded.  Whole warps take part (the encoder exchanges values between the two lanes of a unit): the task
+// count is rounded up to a multiple of 32 and the surplus lanes encode zeros that they do not store.
 template <bool kRHA>
 __device__ __forceinline__ void build_tokens_from_bf16(const uint16_t* __restrict__ X, int64_t ld_x, int M, int64_t upr,
-                                                       uint8_t* tok, int tid, int nthreads) {
-  for (int64_t idx = tid; idx < 16 * upr; idx += nthreads) {      // nthreads is a multiple of 32: warps stay whole
+                                                       uint8_t* tok, int tiles, int rows, int tid, int nthreads) {
+  const int word_bytes = rows * 64;
+  const int64_t tasks = 2 * static_cast<int64_t>(tiles) * rows * upr;
+  for (int64_t idx = tid; idx < ((tasks + 31) & ~static_cast<int64_t>(31)); idx += nthreads) {      // nthreads is a multiple of 32
+    const bool valid = idx < tasks;
     const int l = static_cast<int>(idx & 1);
     const int64_t pair = idx >> 1;
-    const int n = static_cast<int>(pair / upr);
-    const int64_t U = pair - static_cast<int64_t>(n) * upr;
+    const int n = valid ? static_cast<int>(pair / upr) : M;
+    const int64_t U = valid ? pair - static_cast<int64_t>(n) * upr : 0;
+    const int t = n / rows, row = n - t * rows;
     uint4 v[4];
 #pragma unroll
     for (int c = 0; c < 4; ++c) v[c] = make_uint4(0u, 0u, 0u, 0u);
@@ -257,7 +268,8 @@ __device__ __forceinline__ void build_tokens_from_bf16(const uint16_t* __restric
     }
     uint32_t codes[4], meta;
     encode_unit_bf16_pair<kRHA>(v, l, codes, meta);
-    uint8_t* dst = tok + ((U >> 2) * 8) * kTokChunkBytes + ((n & 7) * 4 + (U & 3)) * 16;
+    if (!valid) continue;
+    uint8_t* dst = tok + (((U >> 2) * tiles + t) * 8) * word_bytes + (row * 4 + (U & 3)) * 16;
     const uint32_t byte = meta & 0xFFu;
     const uint32_t base2 = byte * 0x00200020u + 0x26802680u;
 #pragma unroll
@@ -268,7 +280,7 @@ __device__ __forceinline__ void build_tokens_from_bf16(const uint16_t* __restric
         if (byte == 0xFFu) r[0] = r[1] = r[2] = r[3] = 0x7FC07FC0u;
         else decode_word_regs(meta, base2, W, codes[c], r);
       }
-      *reinterpret_cast<uint4*>(dst + W * kTokChunkBytes) = make_uint4(r[0], r[1], r[2], r[3]);
+      *reinterpret_cast<uint4*>(dst + W * word_bytes) = make_uint4(r[0], r[1], r[2], r[3]);
     }
   }
 }
@@ -326,8 +338,11 @@ template <int kTokTiles, int kGemvWarps, int kSrc>
 __global__ void __launch_bounds__((kGemvWarps + 1) * 32, 1)
 gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__ CUtensorMap tm_short, const GemvParams p) {
   constexpr bool kResident = kSrc != kSrcWorkspace;
-  static_assert(!kResident || kTokTiles == 1, "resident tokens: one n-tile");
+  static_assert(!kResident || kTokTiles <= 2, "resident tokens: one or two n-tiles");
   constexpr int kTokBytes = kTokTiles * kTileChunkBytes;
+  // bytes of one word's line of tokens (rows x 4 units x 16 bytes) and of one K = 256 chunk of them
+  const uint32_t tok_word_bytes = kResident ? static_cast<uint32_t>(p.res_rows) * 64u : static_cast<uint32_t>(kTokChunkBytes);
+  const uint32_t tok_chunk_bytes = kTokTiles * 8u * tok_word_bytes;
   constexpr int kRedBytes = kGemvWarps * 32 * 4 * kTokTiles * 4;     // partial accumulators of every consumer warp
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 127u) & ~127u;
@@ -340,7 +355,7 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
   volatile int* announced = reinterpret_cast<volatile int*>(gen_base + 1024 + kRedBytes + 16 * kMaxStages + 16);   // chunk in each stage
   const uint32_t tok_res = bar_base + 384;                              // resident tokens: num_kc chunks of kTokBytes
   uint8_t* tok_res_gen = gen_base + 1024 + kRedBytes + 384;
-  const uint32_t ring = tok_res + (kResident ? static_cast<uint32_t>(p.num_kc) * kTokBytes : 0u);
+  const uint32_t ring = tok_res + (kResident ? static_cast<uint32_t>(p.num_kc) * tok_chunk_bytes : 0u);
   const uint32_t w_bytes_max = static_cast<uint32_t>(p.max_blocks) * kBlockBytes;
   const uint32_t stage_bytes = w_bytes_max + (kResident ? 0 : kTokBytes);
 
@@ -412,13 +427,14 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
     const uint32_t off_lo = static_cast<uint32_t>(16 * pair + g) * kRawRowBytes + q * kUnitBytes;   // MMA row g
     const uint32_t off_hi = off_lo + 8 * kRawRowBytes;                                                // MMA row g + 8
     const uint32_t off_tok = (kResident ? 0u : w_bytes_max) + static_cast<uint32_t>(lane) * 16;
+    const bool tok_row_kept = !kResident || g < p.res_rows;       // resident tokens may keep fewer than eight rows per n-tile
     if (kResident) {
       asm volatile("griddepcontrol.wait;" ::: "memory");      // see the producer
       // every consumer thread helps to build the CTA's own copy of the tokens, then all of them meet
       const int64_t upr = static_cast<int64_t>(p.num_kc) * kRawUnits;
-      if (kSrc == kSrcUnits) build_tokens_from_units(p.A, p.M, upr, tok_res_gen, threadIdx.x, kGemvWarps * 32);
-      else if (p.rha) build_tokens_from_bf16<true>(p.X, p.ld_x, p.M, upr, tok_res_gen, threadIdx.x, kGemvWarps * 32);
-      else build_tokens_from_bf16<false>(p.X, p.ld_x, p.M, upr, tok_res_gen, threadIdx.x, kGemvWarps * 32);
+      if (kSrc == kSrcUnits) build_tokens_from_units(p.A, p.M, upr, tok_res_gen, kTokTiles, p.res_rows, threadIdx.x, kGemvWarps * 32);
+      else if (p.rha) build_tokens_from_bf16<true>(p.X, p.ld_x, p.M, upr, tok_res_gen, kTokTiles, p.res_rows, threadIdx.x, kGemvWarps * 32);
+      else build_tokens_from_bf16<false>(p.X, p.ld_x, p.M, upr, tok_res_gen, kTokTiles, p.res_rows, threadIdx.x, kGemvWarps * 32);
       asm volatile("bar.sync 1, %0;" ::"n"(kGemvWarps * 32) : "memory");
     }
     if (active) {
@@ -430,7 +446,7 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
                                                mbar_wait(full + 8 * s, ph, abort_flag))))
           break;
         const uint32_t st = ring + s * stage_bytes;
-        const uint32_t tk = kResident ? tok_res + static_cast<uint32_t>(kc) * kTokBytes : st;      // this chunk's tokens
+        const uint32_t tk = kResident ? tok_res + static_cast<uint32_t>(kc) * tok_chunk_bytes : st;      // this chunk's tokens
         const uint32_t ml = lds32(st + off_lo), mh = has_hi ? lds32(st + off_hi) : 0u;
         const UnitPrep ul = prepare_unit(ml, lut), uh = prepare_unit(mh, lut);
         // a short loop rather than eight unrolled words: the body stays small enough for the instruction cache
@@ -438,7 +454,8 @@ gemv_kernel(const __grid_constant__ CUtensorMap tm_full, const __grid_constant__
         for (int j = 0; j < 8; ++j) {
           uint4 x[kTokTiles];
 #pragma unroll
-          for (int t = 0; t < kTokTiles; ++t) x[t] = lds128(tk + off_tok + (t * 8 + j) * kTokChunkBytes);
+          for (int t = 0; t < kTokTiles; ++t)
+            x[t] = tok_row_kept ? lds128(tk + off_tok + (t * 8 + j) * tok_word_bytes) : make_uint4(0u, 0u, 0u, 0u);
           uint32_t a[4], b[4] = {0u, 0u, 0u, 0u};
           decode_word(ul, j, lds32(st + off_lo + 4 + 4 * j), p.mul, a);
           if (has_hi) decode_word(uh, j, lds32(st + off_hi + 4 + 4 * j), p.mul, b);
@@ -491,7 +508,7 @@ template <int kTokTiles, int kGemvWarps, int kSrc = kSrcWorkspace>
 hif4_status launch_gemv_t(const void* B, int64_t upr, GemvParams p, cudaStream_t st) {
   constexpr bool kResident = kSrc != kSrcWorkspace;
   constexpr int kTokBytes = kTokTiles * kTileChunkBytes;
-  const int resident_bytes = kResident ? p.num_kc * kTokBytes : 0;
+  const int resident_bytes = kResident ? p.num_kc * kTokTiles * 8 * p.res_rows * 64 : 0;
   constexpr int kFixed = 128 + 1024 + kGemvWarps * 32 * 4 * kTokTiles * 4 + 384;
   // One CTA per SM (several rounds of them when a CTA would get more than kMaxBlocks blocks).
   const int64_t sms = sm_count();
@@ -554,14 +571,26 @@ bool gemv_params(GemvParams& p, float* C, int64_t M, int64_t N, int64_t K, int64
   p.error_word = device_error_word();
   return true;
 }
-// One n-tile of tokens and a K short enough for the tokens to stay in shared memory: the streaming kernel builds them itself.
-bool gemv_tokens_fit_resident(int m_pad, int num_kc) { return m_pad == 8 && num_kc * kTileChunkBytes <= kResidentMaxBytes; }
+// At most two n-tiles of tokens and few enough token elements: the streaming kernel builds them itself, in shared
+// memory.  Returns the token rows kept per n-tile (the next power of two >= M, eight for two tiles), 0 when the
+// two-launch form is the faster one.  Every CTA repeats the build before its main loop, so it pays only while it costs
+// less than the launch it saves: measured break-even (rows kept x K) about 57 000 elements when the tokens are decoded
+// from packed units and about 16 000 when they are first converted from BF16 with Algorithm 1.
+constexpr int64_t kResidentMaxElemsUnits = 49152, kResidentMaxElemsBf16 = 16384;
+int gemv_resident_rows(int64_t M, int num_kc, int64_t max_elems) {
+  if (M > 16) return 0;
+  const int tiles = M <= 8 ? 1 : 2;
+  const int rows = M <= 1 ? 1 : M <= 2 ? 2 : M <= 4 ? 4 : 8;
+  const int64_t elems = static_cast<int64_t>(num_kc) * 256 * tiles * rows;
+  return elems <= max_elems && elems * 2 <= kResidentMaxBytes ? rows : 0;
+}
 template <int kSrc>
 hif4_status launch_gemv_resident(const void* B, const GemvParams& p, int64_t upr, cudaStream_t st) {
   const int64_t sms = sm_count();
   const int64_t rounds = ceil_div64(p.num_blocks, sms * kMaxBlocks);
   const int64_t grid = p.num_blocks < sms * rounds ? p.num_blocks : sms * rounds;
   const bool many = ceil_div64(p.num_blocks, grid) >= 9;
+  if (p.M > 8) return many ? launch_gemv_t<2, kGemvWarpsMany, kSrc>(B, upr, p, st) : launch_gemv_t<2, kGemvWarpsFew, kSrc>(B, upr, p, st);
   return many ? launch_gemv_t<1, kGemvWarpsMany, kSrc>(B, upr, p, st) : launch_gemv_t<1, kGemvWarpsFew, kSrc>(B, upr, p, st);
 }
 // The streaming kernel on tokens that the preceding launch in `st` has prepared.
@@ -585,7 +614,8 @@ hif4_status launch_gemv(const void* A, const void* B, float* C, int64_t M, int64
   if (!p.error_word) return HIF4_ERR_CUDA;
   const int m_pad = static_cast<int>(gemv_m_pad(M));
   const int64_t upr = K / kUnitElems;
-  if (gemv_tokens_fit_resident(m_pad, p.num_kc)) return launch_gemv_resident<kSrcUnits>(B, p, upr, st);     // one launch
+  p.res_rows = gemv_resident_rows(M, p.num_kc, kResidentMaxElemsUnits);
+  if (p.res_rows > 0) return launch_gemv_resident<kSrcUnits>(B, p, upr, st);     // one launch
   const int64_t prep = static_cast<int64_t>(m_pad) * upr;
   gemv_prepare_tokens_kernel<<<static_cast<unsigned>(ceil_div64(prep, 128)), 128, 0, st>>>(p.A, p.M, m_pad, upr, p.tokens);
   note_launch();
@@ -606,7 +636,8 @@ hif4_status launch_gemv_linear(const void* X, hif4_dtype dt, int64_t ld_x, int r
   if (!p.error_word) return HIF4_ERR_CUDA;
   const int m_pad = static_cast<int>(gemv_m_pad(M));
   const int64_t upr = K / kUnitElems;
-  if (dt == HIF4_BF16 && gemv_tokens_fit_resident(m_pad, p.num_kc)) {        // one launch: conversion, decode and streaming
+  p.res_rows = dt == HIF4_BF16 ? gemv_resident_rows(M, p.num_kc, kResidentMaxElemsBf16) : 0;
+  if (p.res_rows > 0) {        // one launch: conversion, decode and streaming
     p.X = static_cast<const uint16_t*>(X); p.ld_x = ld_x; p.rha = rha;
     return launch_gemv_resident<kSrcBf16>(B, p, upr, st);
   }

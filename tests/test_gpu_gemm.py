@@ -6,6 +6,7 @@ import torch
 
 import hif4_workloads as wl
 import oracle
+from tests.kernel_choice import tokens_stay_in_shared_memory
 
 pytestmark = pytest.mark.gpu
 TOL = 1e-5
@@ -359,7 +360,9 @@ def gemv_path(hif4):
                                    (16, 1000, 2304), (16, 64, 4096), (5, 9475, 256), (3, 31, 5120), (12, 77, 14336),
                                    (1, 40003, 256), (16, 2376, 1024), (10, 1192, 512), (4, 19000, 256),
                                    (17, 300, 256), (32, 1000, 1024), (25, 4200, 512), (31, 77, 4096), (20, 14336, 256),
-                                   (8, 300, 6144), (8, 300, 6400), (5, 14336, 4096), (1, 1030, 4096)])
+                                   (8, 300, 6144), (8, 300, 6400), (5, 14336, 4096), (1, 1030, 4096),
+                                   (1, 300, 14336), (2, 300, 14336), (3, 200, 8192), (4, 200, 16384), (8, 300, 8192),
+                                   (8, 300, 8448), (16, 300, 4096), (16, 300, 4352), (12, 14336, 4096), (1, 9, 65536)])
 def test_weight_streaming_kernel_full_compare(gemv_path, M, N, K):
     hif4 = gemv_path
     g = torch.Generator(device="cuda"); g.manual_seed(M * 11 + N)
@@ -369,7 +372,7 @@ def test_weight_streaming_kernel_full_compare(gemv_path, M, N, K):
     before = hif4.launch_count()
     out = torch.full((M + 2, N + 3), -5.0, dtype=torch.float32, device="cuda")
     C = check_full(hif4, a, b, f"gemv {M}x{N}x{K}", out=out[1:M + 1, 1:N + 1])
-    one_launch = M <= 8 and K <= 6144            # few tokens, short K: the streaming kernel decodes the tokens itself
+    one_launch = tokens_stay_in_shared_memory(M, K)      # few tokens, short K: the streaming kernel decodes the tokens itself
     assert hif4.launch_count() - before == (1 if one_launch else 2), "token preparation + streaming kernel, or the latter alone"
     assert (out[0] == -5.0).all() and (out[M + 1] == -5.0).all() and (out[:, 0] == -5.0).all() and (out[:, N + 1:] == -5.0).all()
     C2 = hif4.hif4_gemm(a, b)
@@ -527,10 +530,11 @@ def test_linear_is_quantize_then_gemm(hif4, M, N, K, dtype):
 @pytest.mark.parametrize("mode", [0, 1])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32, torch.float16])
 @pytest.mark.parametrize("M,N,K", [(1, 4096, 4096), (16, 1000, 1024), (7, 260, 256), (9, 64, 2304), (16, 14336, 4096),
-                                   (24, 520, 1024), (32, 64, 256)])
+                                   (24, 520, 1024), (32, 64, 256), (2, 520, 14336), (3, 300, 8192), (13, 300, 4096),
+                                   (2, 300, 4096), (3, 260, 2048), (1, 130, 14336)])
 def test_linear_with_few_rows_quantizes_inside_the_token_preparation(hif4, M, N, K, dtype, mode):
     """M <= 32 rows of activations: hif4_linear runs two kernels (quantize-and-decode of the tokens, weight
-    streaming) instead of three -- a single one for up to eight BF16 rows and K <= 6144 -- and gives exactly the bits
+    streaming) instead of three -- a single one for a few BF16 rows of moderate length -- and gives exactly the bits
     of hif4_quantize followed by hif4_gemm, on a strided source with spikes, a NaN and an Inf, for every source type
     and both rounding modes."""
     g = torch.Generator(device="cuda"); g.manual_seed(M * 3 + N + K + mode)
@@ -543,7 +547,7 @@ def test_linear_with_few_rows_quantizes_inside_the_token_preparation(hif4, M, N,
     w = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
     before = hif4.launch_count()
     y = hif4.hif4_linear(x, w, mode=mode)
-    one_launch = M <= 8 and K <= 6144 and dtype == torch.bfloat16     # conversion, token decode and streaming in one kernel
+    one_launch = dtype == torch.bfloat16 and tokens_stay_in_shared_memory(M, K, from_bf16=True)     # conversion, token decode and streaming in one kernel
     assert hif4.launch_count() - before == (1 if one_launch else 2)
     want = hif4.hif4_gemm(hif4.hif4_quantize(x, mode), w)
     assert torch.equal(y.view(torch.int32), want.view(torch.int32)), "fused token preparation differs from quantize + GEMM"
