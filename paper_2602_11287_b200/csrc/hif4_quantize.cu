@@ -99,6 +99,16 @@ constexpr int kTileCols = 128;
 constexpr int kTileThreads = 64;
 constexpr int kTileRowWords = kTileCols / 2;
 
+// Writes the `ncols` units of a tile (9 words each, one after the other in `units`) to their columns of dst: unit c
+// goes to row tile blockIdx.x of column c0 + c.
+__device__ __forceinline__ void flush_tile_units(const uint32_t* units, uint32_t* __restrict__ dst, int64_t c0, int ncols,
+                                                 int64_t units_per_col) {
+  for (int i = threadIdx.x; i < ncols * kUnitWords; i += kTileThreads) {
+    const int c = i / kUnitWords, w = i - c * kUnitWords;
+    st_stream(dst + ((c0 + c) * units_per_col + blockIdx.x) * kUnitWords + w, units[i]);
+  }
+}
+
 template <bool kRHA>
 __global__ void __launch_bounds__(kTileThreads)
 quantize_bf16_transposed_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t cols, int64_t ld_src,
@@ -109,18 +119,18 @@ quantize_bf16_transposed_kernel(const uint16_t* __restrict__ src, int64_t rows, 
   const int64_t r0 = static_cast<int64_t>(blockIdx.x) * kUnitElems;
   // 64 rows x 16 chunks of 8 elements; a chunk is inside the matrix or outside as a whole (cols % 8 == 0)
   constexpr int kChunks = kUnitElems * (kTileCols / 8) / kTileThreads;      // 16 per thread
-  uint4 in[kChunks];
+  // asynchronous 16-byte copies straight into shared memory (no registers, one instruction per chunk instead of a
+  // load and a store); chunks outside the matrix are filled with zeros
+  const uint32_t tile_addr = static_cast<uint32_t>(__cvta_generic_to_shared(tile));
 #pragma unroll
   for (int n = 0; n < kChunks; ++n) {
-    const int i = n * kTileThreads + threadIdx.x, r = i >> 4, ch = i & 15;
-    in[n] = make_uint4(0u, 0u, 0u, 0u);
-    if (c0 + 8 * ch < cols) in[n] = ld_stream(reinterpret_cast<const uint4*>(src + (r0 + r) * ld_src + c0 + 8 * ch));
+    const int i = n * kTileThreads + threadIdx.x, r = i >> 4, ch = i & 15;           // row i / 16, words 4 (i % 16) ..
+    const bool inside = c0 + 8 * ch < cols;
+    const uint16_t* p = inside ? src + (r0 + r) * ld_src + c0 + 8 * ch : src;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(tile_addr + 16u * i), "l"(p), "r"(inside ? 16 : 0) : "memory");
   }
-#pragma unroll
-  for (int n = 0; n < kChunks; ++n) {
-    const int i = n * kTileThreads + threadIdx.x;
-    *reinterpret_cast<uint4*>(tile + 4 * i) = in[n];                         // row i / 16, words 4 (i % 16) ..
-  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
   const int lane = threadIdx.x & 31, l = lane >> 4;
   const int cq = (threadIdx.x >> 5) * 16 + (lane & 15);                      // columns 4 cq .. 4 cq + 3 of the tile
@@ -142,18 +152,21 @@ quantize_bf16_transposed_kernel(const uint16_t* __restrict__ src, int64_t rows, 
     for (int j = 0; j < 4; ++j) col[j][c] = make_uint4(e[j][0], e[j][1], e[j][2], e[j][3]);
   }
   const int64_t units_per_col = rows / kUnitElems;
+  // The units of neighbouring columns lie a whole column apart in dst: written straight from the encoder's registers,
+  // every 4-byte store of a warp would go to 32 different sectors.  They are collected in the tile's shared memory
+  // instead (all its rows have been read) and written with nine consecutive lanes per unit.
+  __syncthreads();
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     uint32_t codes[4], meta;
     encode_unit_bf16_pair<kRHA, 16>(col[j], l, codes, meta);
-    const int64_t c = c0 + 4 * cq + j;
-    if (c < cols) {
-      uint32_t* out = dst + (c * units_per_col + blockIdx.x) * kUnitWords;
+    uint32_t* out = tile + (4 * cq + j) * kUnitWords;
 #pragma unroll
-      for (int g = 0; g < 4; ++g) st_stream(out + 1 + 2 * g + l, codes[g]);
-      if (l == 0) st_stream(out, meta);
-    }
+    for (int g = 0; g < 4; ++g) out[1 + 2 * g + l] = codes[g];
+    if (l == 0) out[0] = meta;
   }
+  __syncthreads();
+  flush_tile_units(tile, dst, c0, static_cast<int>(cols - c0 < kTileCols ? cols - c0 : kTileCols), units_per_col);
 }
 
 // ----------------------------------------------------------------------------- FP32 quantizer
@@ -216,17 +229,31 @@ quantize_fp32_transposed_kernel(const Src* __restrict__ src, int64_t rows, int64
   const int64_t r0 = static_cast<int64_t>(blockIdx.x) * kUnitElems;
   // 64 rows x 16 chunks of 4 elements; a chunk is inside the matrix or outside as a whole (cols % 8 == 0)
   constexpr int kChunks = kUnitElems * (kTileCols32 / 4) / kTileThreads;    // 16 per thread
-  uint4 in[kChunks];
+  if constexpr (sizeof(Src) == 4) {
+    // FP32 source: asynchronous 16-byte copies straight into shared memory, zeros outside the matrix
+    const uint32_t tile_addr = static_cast<uint32_t>(__cvta_generic_to_shared(tile));
 #pragma unroll
-  for (int n = 0; n < kChunks; ++n) {
-    const int i = n * kTileThreads + threadIdx.x, r = i >> 4, ch = i & 15;
-    in[n] = make_uint4(0u, 0u, 0u, 0u);
-    if (c0 + 4 * ch < cols) in[n] = load_group_fp32(src + (r0 + r) * ld_src + c0 + 4 * ch);
-  }
+    for (int n = 0; n < kChunks; ++n) {
+      const int i = n * kTileThreads + threadIdx.x, r = i >> 4, ch = i & 15;         // row i / 16, words 4 (i % 16) ..
+      const bool inside = c0 + 4 * ch < cols;
+      const Src* p = inside ? src + (r0 + r) * ld_src + c0 + 4 * ch : src;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(tile_addr + 16u * i), "l"(p), "r"(inside ? 16 : 0) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+  } else {
+    uint4 in[kChunks];                                   // FP16 source: widened on the way
 #pragma unroll
-  for (int n = 0; n < kChunks; ++n) {
-    const int i = n * kTileThreads + threadIdx.x;
-    *reinterpret_cast<uint4*>(tile + 4 * i) = in[n];                         // row i / 16, words 4 (i % 16) ..
+    for (int n = 0; n < kChunks; ++n) {
+      const int i = n * kTileThreads + threadIdx.x, r = i >> 4, ch = i & 15;
+      in[n] = make_uint4(0u, 0u, 0u, 0u);
+      if (c0 + 4 * ch < cols) in[n] = load_group_fp32(src + (r0 + r) * ld_src + c0 + 4 * ch);
+    }
+#pragma unroll
+    for (int n = 0; n < kChunks; ++n) {
+      const int i = n * kTileThreads + threadIdx.x;
+      *reinterpret_cast<uint4*>(tile + 4 * i) = in[n];                       // row i / 16, words 4 (i % 16) ..
+    }
   }
   __syncthreads();
   const int lane = threadIdx.x & 31, l = lane >> 3;
@@ -240,6 +267,7 @@ quantize_fp32_transposed_kernel(const Src* __restrict__ src, int64_t rows, int64
       col[0][c][k] = a.x; col[1][c][k] = a.y; col[2][c][k] = a.z; col[3][c][k] = a.w;
     }
   const int64_t units_per_col = rows / kUnitElems;
+  __syncthreads();                                       // the units are collected in the tile's shared memory, as above
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     uint4 v[4];
@@ -247,16 +275,15 @@ quantize_fp32_transposed_kernel(const Src* __restrict__ src, int64_t rows, int64
     for (int c = 0; c < 4; ++c) v[c] = make_uint4(col[j][c][0], col[j][c][1], col[j][c][2], col[j][c][3]);
     uint32_t codes[4], meta;
     encode_unit_fp32_quad<kRHA, 8>(v, l, codes, meta);
-    const int64_t c = c0 + 4 * cq + j;
-    if (c < cols) {
-      uint32_t* out = dst + (c * units_per_col + blockIdx.x) * kUnitWords;
-      if ((l & 1) == 0) {
+    uint32_t* out = tile + (4 * cq + j) * kUnitWords;
+    if ((l & 1) == 0) {
 #pragma unroll
-        for (int g = 0; g < 4; ++g) st_stream(out + 1 + (l >> 1) + 2 * g, codes[g]);
-      }
-      if (l == 0) st_stream(out, meta);
+      for (int g = 0; g < 4; ++g) out[1 + (l >> 1) + 2 * g] = codes[g];
     }
+    if (l == 0) out[0] = meta;
   }
+  __syncthreads();
+  flush_tile_units(tile, dst, c0, static_cast<int>(cols - c0 < kTileCols32 ? cols - c0 : kTileCols32), units_per_col);
 }
 
 template <typename Src>

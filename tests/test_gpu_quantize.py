@@ -213,7 +213,7 @@ def test_quantize_transposed_is_quantize_of_the_transpose(hif4, mode):
     counts, a strided source, random bit patterns (NaN and Inf included) and the workload mix."""
     rng = np.random.default_rng(500 + mode)
     cases = []
-    for (rows, cols) in ((64, 8), (128, 72), (640, 1000), (1024, 2048)):
+    for (rows, cols) in ((64, 8), (128, 72), (192, 136), (640, 1000), (1024, 2048), (448, 264)):
         expo = rng.integers(100, 150, size=(1, cols), dtype=np.uint32)                 # per column: base exponent
         mant = rng.integers(0, 1 << 7, size=(rows, cols), dtype=np.uint32)
         sign = rng.integers(0, 2, size=(rows, cols), dtype=np.uint32) << 15
@@ -231,10 +231,10 @@ def test_quantize_transposed_is_quantize_of_the_transpose(hif4, mode):
         assert (out[0] == 0xCD).all() and (out[cols + 1] == 0xCD).all()
         assert torch.equal(out[1:cols + 1], hif4.hif4_quantize(x.t().contiguous(), mode)), "differs from quantizing the transpose"
     # strided source
-    wide = wl.u16_numpy_to_bf16(cases[2], "cuda")
+    wide = wl.u16_numpy_to_bf16(cases[3], "cuda")
     view = wide[:, 8:808]
     got = hif4.hif4_quantize_transposed(view, mode).cpu().numpy()
-    _compare_units(got, oracle.quantize(np.ascontiguousarray(cases[2][:, 8:808].T), mode, nthreads=8), "transposed, strided")
+    _compare_units(got, oracle.quantize(np.ascontiguousarray(cases[3][:, 8:808].T), mode, nthreads=8), "transposed, strided")
     # argument checks
     with pytest.raises(hif4.Hif4Error) as ei:
         hif4.hif4_quantize_transposed(torch.zeros(100, 64, dtype=torch.bfloat16, device="cuda"))
@@ -254,7 +254,7 @@ def test_quantize_transposed_fp32_and_fp16_sources(hif4, mode, dtype):
     rng = np.random.default_rng(900 + mode)
     np_dt = np.float32 if dtype == torch.float32 else np.float16
     cases = []
-    for (rows, cols) in ((64, 8), (128, 72), (640, 1000), (512, 2048)):
+    for (rows, cols) in ((64, 8), (128, 72), (192, 136), (640, 1000), (512, 2048), (448, 264)):
         scale = np.exp2(rng.integers(-12, 12, size=(1, cols))) if dtype == torch.float32 else np.exp2(rng.integers(-6, 6, size=(1, cols)))
         x = rng.standard_normal((rows, cols)) * scale * np.exp2(-rng.integers(0, 6, size=(rows, cols)))
         cases.append(x.astype(np_dt))
@@ -271,7 +271,7 @@ def test_quantize_transposed_fp32_and_fp16_sources(hif4, mode, dtype):
         _compare_units(out[1:cols + 1].cpu().numpy(), want, f"transposed {dtype} {rows}x{cols} mode {mode}")
         assert (out[0] == 0xCD).all() and (out[cols + 1] == 0xCD).all()
         assert torch.equal(out[1:cols + 1], hif4.hif4_quantize(x.t().contiguous(), mode)), "differs from quantizing the transpose"
-    wide = torch.from_numpy(cases[2]).cuda()
+    wide = torch.from_numpy(cases[3]).cuda()
     got = hif4.hif4_quantize_transposed(wide[:, 8:808], mode).cpu().numpy()
-    _compare_units(got, oracle.quantize(np.ascontiguousarray(cases[2][:, 8:808].T), mode, nthreads=8), "transposed, strided")
+    _compare_units(got, oracle.quantize(np.ascontiguousarray(cases[3][:, 8:808].T), mode, nthreads=8), "transposed, strided")
     assert hif4.hif4_last_device_status() == 0
