@@ -348,7 +348,7 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
             if (col_ok && tok + v < un.tok_end) {
               float* dst = cp + static_cast<int64_t>(v) * p.ldc;
               if (adds) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst), "f"(__uint_as_float(r[v])) : "memory");
-              else *dst = __uint_as_float(r[v]);
+              else __stcs(dst, __uint_as_float(r[v]));       // C is written once and not read again by this kernel
             }
         }
       }
