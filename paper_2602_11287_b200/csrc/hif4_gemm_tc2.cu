@@ -567,7 +567,9 @@ static hif4_status launch_gemm_tc2_any(const void* A, const uint16_t* x, int64_t
   if (!p.error_word) return HIF4_ERR_CUDA;
   p.mul = make_decode_mul();
   CUtensorMap tmC = tmA;                              // placeholder when the store path is not used
-  p.tma_store = ((reinterpret_cast<uintptr_t>(C) & 15u) == 0 && ldc % 4 == 0 && make_c_map(&tmC, C, M, N, ldc)) ? 1 : 0;
+  // (a TMA store clips the innermost dimension in 16-byte pieces: with N % 4 != 0 it would write up to three columns
+  // past N, so such shapes take the per-thread stores)
+  p.tma_store = ((reinterpret_cast<uintptr_t>(C) & 15u) == 0 && ldc % 4 == 0 && N % 4 == 0 && make_c_map(&tmC, C, M, N, ldc)) ? 1 : 0;
   const Tc2Plan pl = tc2_plan(M, N, K);
   p.full_rounds = pl.full_rounds;
   p.tail_tiles = pl.tail_tiles;

@@ -85,6 +85,38 @@ def test_random_units_all_scales_and_strided_c(hif4):
     assert (out[:, N:] == -5.0).all()
 
 
+@pytest.mark.parametrize("M,N,ld,K", [(300, 90, 96, 256), (300, 257, 260, 512), (513, 258, 260, 256), (300, 259, 260, 256),
+                                      (70, 90, 96, 256), (128, 1030, 1032, 1024), (16, 90, 96, 256), (2500, 1298, 1300, 1280),
+                                      (1000, 4098, 4100, 512)])
+def test_c_inside_a_wider_buffer_with_a_column_count_that_is_not_a_multiple_of_four(hif4, M, N, ld, K):
+    """C as the left columns of a wider, 16-byte aligned buffer (ldc % 4 == 0) with N % 4 != 0: a store path that clips
+    in 16-byte pieces would write the columns between N and the next multiple of four.  Nothing right of column N may
+    change, on any kernel (pair kernel with whole and shared tiles, swapped pair kernel, weight streaming)."""
+    g = torch.Generator(device="cuda"); g.manual_seed(M + N)
+    a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
+    b = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
+    out = torch.full((M + 2, ld), -5.0, dtype=torch.float32, device="cuda")
+    check_full(hif4, a, b, f"{M}x{N} in a buffer of {ld} columns", out=out[1:M + 1, :N])
+    assert (out[:, N:] == -5.0).all() and (out[0] == -5.0).all() and (out[M + 1] == -5.0).all()
+    assert hif4.hif4_last_device_status() == 0
+
+
+def test_grouped_c_inside_a_wider_buffer_with_a_column_count_that_is_not_a_multiple_of_four(hif4):
+    rng = np.random.default_rng(23)
+    counts = [300, 0, 17, 64, 130]
+    total, N, ld, upr = sum(counts), 90, 96, 4
+    A = rng.integers(0, 256, (total, upr, 36), dtype=np.uint8)
+    B = rng.integers(0, 256, (len(counts), N, upr, 36), dtype=np.uint8)
+    A[..., 0] = rng.integers(0x60, 0xE0, (total, upr)); B[..., 0] = rng.integers(0x60, 0xE0, (len(counts), N, upr))
+    off_h = np.concatenate([[0], np.cumsum(counts)]).astype(np.int64)
+    out = torch.full((total + 2, ld), -5.0, dtype=torch.float32, device="cuda")
+    C = hif4.hif4_grouped_gemm(torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), torch.from_numpy(off_h).cuda(),
+                               out=out[1:total + 1, :N])
+    ref, refabs = oracle.grouped_gemm_f64(A, B, off_h, nthreads=8)
+    assert np.all(np.abs(C.cpu().numpy().astype(np.float64) - ref) <= TOL * refabs + 1e-300)
+    assert (out[:, N:] == -5.0).all() and (out[0] == -5.0).all() and (out[total + 1] == -5.0).all()
+
+
 def test_nan_units_and_determinism(hif4):
     rng = np.random.default_rng(22)
     A = rng.integers(0, 256, (66, 4, 36), dtype=np.uint8); A[..., 0] = 0xC0
