@@ -45,7 +45,9 @@ constexpr int kTokThreads = 128;                               // (unit of the c
 constexpr int kSmallT = 64;                                    // token tiles up to this many rows take two weight tiles
 constexpr int kTokBufBytes = 32 * 128;                         // decoded token rows of one K = 64 block (small mode)
 constexpr int kThreads = kDecodeWarp0 * 32 + kDecodeThreads + kTokThreads;   // 832
+constexpr int kEpiBufBytes = 16 * 32 * 4;                      // epilogue staging of one warp: 16 token rows x 32 columns of C
 constexpr int kSmemBytes = 1024 + kDecStages * kDecStageBytes + kRawStages * kRawStageBytes + kDecStages * kTokBufBytes + 256 + 1024;
+constexpr int kSmemBytesStaged = kSmemBytes + 4 * kEpiBufBytes;
 
 // tcgen05.mma kind::f16 descriptor without the N field: D = F32, A = B = BF16, K-major, M = 256.
 constexpr uint32_t kInstrDescM256 = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(256 >> 4) << 24);
@@ -192,15 +194,26 @@ __device__ __noinline__ bool wait_word(const unsigned int* word, unsigned int wa
   }
 }
 
+// kStagedEpi: the epilogue passes C through a staging block in shared memory (see there); the other instantiation
+// stores straight from the accumulator registers.  Two kernels rather than one with both paths: records with a long K
+// gain nothing from the staged form and keep the smaller kernel.  What only the staged epilogue needs rides behind
+// the common parameters, so that the other instantiation's parameter block keeps its layout.
+template <bool kStagedEpi> struct EpilogueArgs {};
+template <> struct EpilogueArgs<true> {
+  CUtensorMap tmC;          // FP32 view of C, box = 32 columns x 16 rows
+  int tma_store;            // 1: whole 16-row chunks of C go out through tmC
+};
+template <bool kStagedEpi>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constant__ CUtensorMap tmW,
-                 const GroupedParams p) {
+                 const GroupedParams p, const __grid_constant__ EpilogueArgs<kStagedEpi> epi) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t dec_base = smem_base;                                        // 1024-byte aligned stages
   const uint32_t raw_base = dec_base + kDecStages * kDecStageBytes;
   const uint32_t tok_base = raw_base + kRawStages * kRawStageBytes;        // 1024-byte aligned: small-mode token blocks
-  const uint32_t bar_base = tok_base + kDecStages * kTokBufBytes;
+  const uint32_t epi_base = tok_base + kDecStages * kTokBufBytes;          // 1024-byte aligned: epilogue staging, one block per warp
+  const uint32_t bar_base = epi_base + (kStagedEpi ? 4 * kEpiBufBytes : 0);
   const uint32_t raw_full = bar_base, raw_empty = bar_base + 16, dec_full = bar_base + 32, dec_empty = bar_base + 64,
                  tmem_full = bar_base + 96, tmem_empty = bar_base + 112;
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -315,6 +328,7 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
     // ---------------------------------------------------------------- epilogue: C^T tile -> rows of C
     const int q = warp & 3;                      // TMEM lane quadrant this warp may read
     const uint32_t tmem_empty_leader = mapa(tmem_empty, 0);
+    [[maybe_unused]] const uint32_t my_buf = epi_base + static_cast<uint32_t>(q) * kEpiBufBytes;
     uint32_t ucount = 0;
     for (int u = pair; u < total_units; u += num_pairs) {
       const Unit un = unit_of(p, u);
@@ -341,24 +355,59 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + 8 * acc);
           }
-          const int tok = un.tok0 + c * 16;
-          float* cp = p.C + static_cast<int64_t>(tok) * p.ldc + col;
+          if constexpr (kStagedEpi) {
+            const int tok = un.tok0 + c * 16;
+            // The lanes put their column of the 16 x 32 chunk into the warp's staging block (row v = 32 consecutive
+            // floats: no bank conflicts).  A chunk whose sixteen token rows all exist then goes out as one TMA store,
+            // which also clips columns past N; the last rows of a group, a C that the tensor map cannot describe and the
+            // adding slices of a K-sliced tile are written row by row from the block (each lane its own column) -- a
+            // short rolled loop instead of sixteen tested, 64-bit-addressed stores per lane in the instruction stream.
+            const int64_t col0 = static_cast<int64_t>(un.n0) + a * 256 + rank * kWRows + q * 32;
+            const int n_rows = un.tok_end - tok < 16 ? un.tok_end - tok : 16;        // warp-uniform, may be <= 0
+            if (col0 >= p.N || n_rows <= 0) continue;
+            if (lane == 0) bulk_wait_read<0>();        // the previous TMA store has read the block
+            __syncwarp();
 #pragma unroll
-          for (int v = 0; v < 16; ++v)
-            if (col_ok && tok + v < un.tok_end) {
-              float* dst = cp + static_cast<int64_t>(v) * p.ldc;
-              if (adds) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst), "f"(__uint_as_float(r[v])) : "memory");
-              else __stcs(dst, __uint_as_float(r[v]));       // C is written once and not read again by this kernel
+            for (int v = 0; v < 16; ++v)
+              asm volatile("st.shared.u32 [%0], %1;" ::"r"(my_buf + static_cast<uint32_t>(v * 128 + lane * 4)), "r"(r[v]) : "memory");
+            if (epi.tma_store && !adds && n_rows == 16) {
+              fence_proxy_async_smem();
+              __syncwarp();
+              if (lane == 0) {
+                tma_store_2d(&epi.tmC, static_cast<int>(col0), tok, my_buf);
+                bulk_commit();
+              }
+            } else if (col_ok) {
+              float* cp = p.C + static_cast<int64_t>(tok) * p.ldc + col;
+#pragma unroll 1
+              for (int v = 0; v < n_rows; ++v, cp += p.ldc) {
+                const float x = __uint_as_float(lds32(my_buf + static_cast<uint32_t>(v * 128 + lane * 4)));
+                if (adds) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(cp), "f"(x) : "memory");
+                else __stcs(cp, x);                  // C is written once and not read again by this kernel
+              }
             }
+          } else {
+            const int tok = un.tok0 + c * 16;
+            float* cp = p.C + static_cast<int64_t>(tok) * p.ldc + col;
+#pragma unroll
+            for (int v = 0; v < 16; ++v)
+              if (col_ok && tok + v < un.tok_end) {
+                float* dst = cp + static_cast<int64_t>(v) * p.ldc;
+                if (adds) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst), "f"(__uint_as_float(r[v])) : "memory");
+                else __stcs(dst, __uint_as_float(r[v]));       // C is written once and not read again by this kernel
+              }
+          }
         }
       }
       if (p.slices > 1 && un.slice + 1 < p.slices) {      // the next slice may add to these columns now
+        if (kStagedEpi && lane == 0) bulk_wait_all();     // (its own stores, if any went through the tensor map, have landed)
         __threadfence();
         __syncwarp();
         if (lane == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(my_flag), "r"(1u) : "memory");
       }
       ++ucount;
     }
+    if (kStagedEpi && lane == 0) bulk_wait_all();  // shared memory stays valid until the last store has read it
   } else if (warp >= kTokWarp0) {
     // ---------------------------------------------------------------- token warps (small-tile mode): warp w = unit w of the chunk
     const int w = warp - kTokWarp0;
@@ -453,10 +502,24 @@ gemm_tc2g_kernel(const __grid_constant__ CUtensorMap tmTok, const __grid_constan
   }
 }
 
+// FP32 view of C [rows, N] for the epilogue's TMA stores: box = 32 columns x 16 rows.
+bool make_c_map_g(CUtensorMap* map, float* C, int64_t rows, int64_t N, int64_t ldc) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ldc) * 4};
+  const cuuint32_t box[2] = {32, 16};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 hif4_status launch_swapped(const void* A, const void* B, int64_t a_rows, int64_t b_rows, GroupedParams p, int64_t K,
                            cudaStream_t st) {
-  static uint64_t smem_opt_in = 0;
-  if (!ensure_dynamic_smem(gemm_tc2g_kernel, kSmemBytes, smem_opt_in)) return HIF4_ERR_CUDA;
+  static uint64_t smem_opt_in = 0, smem_opt_in_staged = 0;
+  if (!ensure_dynamic_smem(gemm_tc2g_kernel<false>, kSmemBytes, smem_opt_in) ||
+      !ensure_dynamic_smem(gemm_tc2g_kernel<true>, kSmemBytesStaged, smem_opt_in_staged))
+    return HIF4_ERR_CUDA;
   CUtensorMap tmTok, tmW;
   const int64_t upr = K / kUnitElems;
   if (!make_unit_map(&tmTok, A, a_rows, upr, 128) || !make_unit_map(&tmW, B, b_rows, upr, kWRows)) return HIF4_ERR_CUDA;
@@ -470,7 +533,19 @@ hif4_status launch_swapped(const void* A, const void* B, int64_t a_rows, int64_t
   const int64_t units = static_cast<int64_t>(p.max_entries) * p.n_wtiles * p.slices;
   if (units > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
   const int pairs = static_cast<int>(units < sm_count() / 2 ? units : sm_count() / 2);
-  gemm_tc2g_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tmTok, tmW, p);
+  // The staged epilogue where a record is short (at most 16 K chunks), i.e. where the epilogue's instructions weigh
+  // against the main loop's: K = 2048 grouped 1095 -> 959 us (full token tiles), dense M = 128, N = K = 4096 34.9 ->
+  // 30.8 us; long records (K = 7168 grouped) gain nothing from it.  Its TMA stores need a C that a tensor map can
+  // describe; a TMA store clips the innermost dimension in 16-byte pieces, so N must be a multiple of four columns.
+  if (ceil_div64(p.num_kc, p.slices) <= 16) {
+    EpilogueArgs<true> epi;
+    epi.tmC = tmW;                                    // placeholder when the store path is not used
+    epi.tma_store = ((reinterpret_cast<uintptr_t>(p.C) & 15u) == 0 && p.ldc % 4 == 0 && p.N % 4 == 0 && a_rows < (1ll << 31) &&
+                     make_c_map_g(&epi.tmC, p.C, a_rows, p.N, p.ldc)) ? 1 : 0;
+    gemm_tc2g_kernel<true><<<2 * pairs, kThreads, kSmemBytesStaged, st>>>(tmTok, tmW, p, epi);
+  } else {
+    gemm_tc2g_kernel<false><<<2 * pairs, kThreads, kSmemBytes, st>>>(tmTok, tmW, p, EpilogueArgs<false>{});
+  }
   note_launch();
   return launch_status();
 }
