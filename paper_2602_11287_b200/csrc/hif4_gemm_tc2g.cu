@@ -533,11 +533,14 @@ hif4_status launch_swapped(const void* A, const void* B, int64_t a_rows, int64_t
   const int64_t units = static_cast<int64_t>(p.max_entries) * p.n_wtiles * p.slices;
   if (units > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
   const int pairs = static_cast<int>(units < sm_count() / 2 ? units : sm_count() / 2);
-  // The staged epilogue where a record is short (at most 16 K chunks), i.e. where the epilogue's instructions weigh
-  // against the main loop's: K = 2048 grouped 1095 -> 959 us (full token tiles), dense M = 128, N = K = 4096 34.9 ->
-  // 30.8 us; long records (K = 7168 grouped) gain nothing from it.  Its TMA stores need a C that a tensor map can
-  // describe; a TMA store clips the innermost dimension in 16-byte pieces, so N must be a multiple of four columns.
-  if (ceil_div64(p.num_kc, p.slices) <= 16) {
+  // The staged epilogue where it pays (ncu durations, staged against plain stores).  A dense problem has about one
+  // record per pair, so its epilogue is not hidden behind a next main loop: M = 128, N = K = 4096 30.9 vs 33.3 us,
+  // N = 14336 38.0 vs 41.1 us, M = 64 36.3 vs 37.4 us.  A grouped problem hides the epilogue and gains only while its
+  // instructions weigh against a short main loop: K = 2048 -12 %, K = 2560 -4.6 %, K = 3072 equal, K = 4096 +1 %,
+  // K = 5120 +2 %, K = 7168 +3 to +6 % (the staging adds to the shared-memory pipe, which the main loop owns there).
+  // The TMA stores need a C that a tensor map can describe; a TMA store clips the innermost dimension in 16-byte pieces,
+  // so N must be a multiple of four columns.
+  if (p.table == nullptr || ceil_div64(p.num_kc, p.slices) <= 10) {
     EpilogueArgs<true> epi;
     epi.tmC = tmW;                                    // placeholder when the store path is not used
     epi.tma_store = ((reinterpret_cast<uintptr_t>(p.C) & 15u) == 0 && p.ldc % 4 == 0 && p.N % 4 == 0 && a_rows < (1ll << 31) &&
