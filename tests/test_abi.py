@@ -104,3 +104,21 @@ def test_argument_errors_are_found_before_any_launch(cdll):
     assert cdll.hif4_gemm(None, None, None, 4, 4, 100, 4, None, 0, None) == 2
     assert cdll.hif4_gemm(None, None, None, 0, 4, 64, 4, None, 0, None) == 0
     assert cdll.hif4_debug_launch_count() == before
+
+
+def test_launch_count_helper_of_the_tests_states_the_limits_of_the_source():
+    """tests/kernel_choice.py restates, for the launch-count expectations of the GPU tests, when the weight-streaming
+    kernel builds its tokens itself; its numbers must be the ones compiled into the library."""
+    import re
+    from tests.kernel_choice import tokens_stay_in_shared_memory
+    src = open(os.path.join(ROOT, "paper_2602_11287_b200", "csrc", "hif4_gemv.cu")).read()
+    units = int(re.search(r"kResidentMaxElemsUnits = (\d+)", src).group(1))
+    bf16 = int(re.search(r"kResidentMaxElemsBf16 = (\d+)", src).group(1))
+    max_bytes = int(re.search(r"kResidentMaxBytes = (\d+) \* 1024", src).group(1)) * 1024
+    assert min(units, bf16) * 2 <= max_bytes
+    for (M, rows) in ((1, 1), (2, 2), (3, 4), (4, 4), (5, 8), (8, 8), (9, 16), (16, 16)):
+        for limit, from_bf16 in ((units, False), (bf16, True)):
+            k_fit = limit // rows // 256 * 256
+            if k_fit * rows * 2 <= max_bytes:
+                assert tokens_stay_in_shared_memory(M, k_fit, from_bf16) and not tokens_stay_in_shared_memory(M, k_fit + 256, from_bf16)
+    assert not tokens_stay_in_shared_memory(17, 256)
