@@ -81,12 +81,18 @@ struct GroupedParams {
 
 // Work table from the device-side offsets: every group is cut into token tiles of 256 rows, the last one padded
 // to a multiple of 32; a tile of more than kSmallT rows gives one record per 256 weight rows, a smaller one a
-// record per PAIR of weight tiles.  Thread g counts the records of group g, a block-wide scan places them, the
-// thread writes them; groups are taken 256 at a time.
+// record per PAIR of weight tiles.  Thread g counts the records of group g and a block-wide scan places them; then
+// the records of the 256 groups are written as one flat list, record i by thread i % 256 of block (i / 256) % blocks
+// (it finds the group of a record by bisection in the scanned counts), so a hot expert's hundreds of records cost no
+// more than anyone else's.  Every block repeats the counting and the scan (a few microseconds) and writes its share
+// of the list; block 0 writes the record count.  Groups are taken 256 at a time.
+constexpr int kTableBlocks = 16;
 __global__ void __launch_bounds__(256)
 build_work_table_kernel(const int64_t* __restrict__ offsets, int num_groups, int64_t N, int n_wtiles, uint8_t* table_mem,
                         int max_records) {
   __shared__ int warp_sums[8];
+  __shared__ int s_first[257];                 // first record of each group of the batch (relative), and their total
+  __shared__ int64_t s_lo[256], s_hi[256];
   __shared__ int s_base;
   WorkRec* table = reinterpret_cast<WorkRec*>(table_mem + kTableHeaderBytes);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -96,7 +102,8 @@ build_work_table_kernel(const int64_t* __restrict__ offsets, int num_groups, int
     const int g = g0 + threadIdx.x;
     int64_t lo = 0, hi = 0;
     if (g < num_groups) { lo = offsets[g]; hi = offsets[g + 1]; }
-    const int64_t rows = hi > lo ? hi - lo : 0;
+    if (hi < lo) hi = lo;
+    const int64_t rows = hi - lo;
     const int64_t full = rows / kMaxTok;
     const int rest = static_cast<int>(rows - full * kMaxTok);
     const int rest_units = rest == 0 ? 0 : rest <= kSmallT ? (n_wtiles + 1) / 2 : n_wtiles;
@@ -110,28 +117,45 @@ build_work_table_kernel(const int64_t* __restrict__ offsets, int num_groups, int
     }
     if (lane == 31) warp_sums[warp] = incl;
     __syncthreads();
-    int before = s_base;
+    int before = 0;
     for (int w = 0; w < warp; ++w) before += warp_sums[w];
-    int n = before + incl - mine;
-    for (int64_t r = lo; r < hi; r += kMaxTok) {
-      const int t_rows = static_cast<int>(hi - r < kMaxTok ? hi - r : kMaxTok);
-      const int step = t_rows <= kSmallT ? 2 : 1;
-      for (int wt = 0; wt < n_wtiles && n < max_records; wt += step, ++n) {
-        WorkRec rec;
-        rec.tok0 = static_cast<int>(r);
-        rec.tok_end = static_cast<int>(hi);
-        rec.n0 = wt * 256;
-        rec.w_row0 = static_cast<int>(g * N) + rec.n0;
-        rec.T = (t_rows + 31) & ~31;
-        rec.tiles = step == 2 ? (wt + 1 < n_wtiles ? 2 : 3) : 1;       // 3: small-tile mode whose second weight tile does not exist
-        table[n] = rec;
+    s_first[threadIdx.x] = before + incl - mine;
+    if (threadIdx.x == 255) s_first[256] = before + incl;
+    s_lo[threadIdx.x] = lo; s_hi[threadIdx.x] = hi;
+    __syncthreads();
+    const int batch_total = s_first[256], base = s_base;
+    for (int i = blockIdx.x * 256 + threadIdx.x; i < batch_total && base + i < max_records; i += 256 * gridDim.x) {
+      int a = 0, b = 256;                               // the last group whose first record is <= i (empty groups skipped)
+      while (b - a > 1) {
+        const int m = (a + b) >> 1;
+        if (s_first[m] <= i) a = m; else b = m;
       }
+      const int64_t g_lo = s_lo[a], g_hi = s_hi[a];
+      const int j = i - s_first[a];
+      const int g_full = static_cast<int>((g_hi - g_lo) / kMaxTok), g_rest = static_cast<int>((g_hi - g_lo) - static_cast<int64_t>(g_full) * kMaxTok);
+      WorkRec rec;
+      int t_rows, wt, step;
+      if (j < g_full * n_wtiles) {                        // a whole token tile
+        const int tile = j / n_wtiles;
+        wt = j - tile * n_wtiles; step = 1; t_rows = kMaxTok;
+        rec.tok0 = static_cast<int>(g_lo + static_cast<int64_t>(tile) * kMaxTok);
+      } else {                                          // the last tile of the group
+        step = g_rest <= kSmallT ? 2 : 1;
+        wt = (j - g_full * n_wtiles) * step; t_rows = g_rest;
+        rec.tok0 = static_cast<int>(g_lo + static_cast<int64_t>(g_full) * kMaxTok);
+      }
+      rec.tok_end = static_cast<int>(g_hi);
+      rec.n0 = wt * 256;
+      rec.w_row0 = static_cast<int>(static_cast<int64_t>(g0 + a) * N) + rec.n0;
+      rec.T = (t_rows + 31) & ~31;
+      rec.tiles = step == 2 ? (wt + 1 < n_wtiles ? 2 : 3) : 1;       // 3: small-tile mode whose second weight tile does not exist
+      table[base + i] = rec;
     }
     __syncthreads();
-    if (threadIdx.x == 255) s_base = before + incl;
+    if (threadIdx.x == 0) s_base = base + batch_total;
     __syncthreads();
   }
-  if (threadIdx.x == 0) *reinterpret_cast<int*>(table_mem) = s_base < max_records ? s_base : max_records;
+  if (blockIdx.x == 0 && threadIdx.x == 0) *reinterpret_cast<int*>(table_mem) = s_base < max_records ? s_base : max_records;
 }
 
 struct Unit { int tok0; int tok_end; int T; int w_row0; int n0; int kc0; int kc1; int wt; int slice; int tiles; };
@@ -606,7 +630,7 @@ hif4_status launch_grouped_gemm_tc2(const void* A, const void* B, float* C, cons
   const int64_t max_records = (ceil_div64(total_rows, kMaxTok) + num_groups) * n_wtiles;
   if (max_records > 0x7FFFFFFFll) return HIF4_ERR_SHAPE;
   uint8_t* table_mem = static_cast<uint8_t*>(workspace);
-  build_work_table_kernel<<<1, 256, 0, st>>>(offsets, num_groups, N, n_wtiles, table_mem, static_cast<int>(max_records));
+  build_work_table_kernel<<<kTableBlocks, 256, 0, st>>>(offsets, num_groups, N, n_wtiles, table_mem, static_cast<int>(max_records));
   note_launch();
   if (cudaGetLastError() != cudaSuccess) return HIF4_ERR_CUDA;
   GroupedParams p{};
