@@ -87,11 +87,13 @@ def test_random_units_all_scales_and_strided_c(hif4):
 
 @pytest.mark.parametrize("M,N,ld,K", [(300, 90, 96, 256), (300, 257, 260, 512), (513, 258, 260, 256), (300, 259, 260, 256),
                                       (70, 90, 96, 256), (128, 1030, 1032, 1024), (16, 90, 96, 256), (2500, 1298, 1300, 1280),
-                                      (1000, 4098, 4100, 512)])
+                                      (1000, 4098, 4100, 512), (70, 24, 28, 256), (100, 8, 8, 512), (128, 36, 40, 256),
+                                      (300, 8, 12, 256)])
 def test_c_inside_a_wider_buffer_with_a_column_count_that_is_not_a_multiple_of_four(hif4, M, N, ld, K):
     """C as the left columns of a wider, 16-byte aligned buffer (ldc % 4 == 0) with N % 4 != 0: a store path that clips
     in 16-byte pieces would write the columns between N and the next multiple of four.  Nothing right of column N may
-    change, on any kernel (pair kernel with whole and shared tiles, swapped pair kernel, weight streaming)."""
+    change, on any kernel (pair kernel with whole and shared tiles, swapped pair kernel, weight streaming).  The last
+    shapes have fewer columns than the store boxes are wide."""
     g = torch.Generator(device="cuda"); g.manual_seed(M + N)
     a = hif4.hif4_quantize(torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16))
     b = hif4.hif4_quantize((torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16))
